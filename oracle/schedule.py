@@ -1,0 +1,91 @@
+"""The paper's tile schedule, written out in plain Python (test infrastructure).
+
+Algorithm 2 (persistent CTAs, grid-stride loop): G = min(N_tiles, N_SM) CTAs; CTA c handles the
+linear work indices k = c, c + G, c + 2G, ... while k < N_tiles.  Each k names one
+(batch, head, Q tile).  The paper does not say which of the three varies fastest; here the Q tile
+does, then the head, then the batch ("tile_fastest"), so that CTAs running side by side stream
+the K/V of the same head, which is the reuse between wavefronts that the paper observes.
+"head_fastest" is the alternative order (head, then Q tile, then batch).
+
+Algorithm 4 (sawtooth): every CTA counts the Q tiles it has handled so far (i_local).  On an even
+count it scans its K/V tiles from the first to the last, on an odd count from the last to the
+first.  The cyclic order always scans from the first to the last.
+
+Causal mask: Q tile t (rows t*W .. min(N,(t+1)*W)-1) needs K/V tiles 0 .. hi-1 with
+hi = ceil(min(N,(t+1)*W) / B_c); the tiles beyond are never visited, in either direction.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Iterator
+
+CYCLIC = 0
+SAWTOOTH = 1
+
+
+@dataclass(frozen=True)
+class WorkItem:
+    cta: int
+    i_local: int
+    k: int
+    batch: int
+    head: int
+    q_tile: int
+    backward: bool
+    n_kv: int  # K/V tiles this Q tile visits (0 .. n_kv-1)
+
+    def kv_order(self) -> range:
+        return range(self.n_kv - 1, -1, -1) if self.backward else range(self.n_kv)
+
+
+def ceil_div(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+def grid_size(n_tiles: int, n_sm: int) -> int:
+    """Algorithm 2: one persistent CTA per SM, never more CTAs than Q tiles."""
+    return min(n_tiles, n_sm)
+
+
+def decode(k: int, B: int, H: int, n_q: int, digit_order: str = "tile_fastest") -> tuple[int, int, int]:
+    """Linear work index -> (batch, head, Q tile)."""
+    if digit_order == "tile_fastest":
+        t = k % n_q
+        h = (k // n_q) % H
+        b = k // (n_q * H)
+    elif digit_order == "head_fastest":
+        h = k % H
+        t = (k // H) % n_q
+        b = k // (n_q * H)
+    else:
+        raise ValueError(digit_order)
+    return b, h, t
+
+
+def kv_tiles_needed(t: int, N: int, W: int, B_c: int, causal: bool) -> int:
+    if not causal:
+        return ceil_div(N, B_c)
+    last_row_excl = min(N, (t + 1) * W)
+    return ceil_div(last_row_excl, B_c)
+
+
+def cta_sequence(cta: int, G: int, B: int, H: int, N: int, W: int, B_c: int, causal: bool,
+                 scan_order: int, digit_order: str = "tile_fastest") -> Iterator[WorkItem]:
+    """The Q tiles one CTA handles, in order, each with its K/V scan (Algorithms 2 and 4)."""
+    n_q = ceil_div(N, W)
+    n_tiles = B * H * n_q
+    i_local = 0
+    k = cta
+    while k < n_tiles:
+        b, h, t = decode(k, B, H, n_q, digit_order)
+        backward = scan_order == SAWTOOTH and i_local % 2 == 1
+        yield WorkItem(cta, i_local, k, b, h, t, backward, kv_tiles_needed(t, N, W, B_c, causal))
+        i_local += 1
+        k += G
+
+
+def full_schedule(n_sm: int, B: int, H: int, N: int, W: int, B_c: int, causal: bool,
+                  scan_order: int, digit_order: str = "tile_fastest", max_ctas: int = 0) -> list[list[WorkItem]]:
+    n_tiles = B * H * ceil_div(N, W)
+    G = grid_size(n_tiles, n_sm if max_ctas <= 0 else min(n_sm, max_ctas))
+    return [list(cta_sequence(c, G, B, H, N, W, B_c, causal, scan_order, digit_order)) for c in range(G)]
