@@ -1,0 +1,150 @@
+/*
+ * sawtooth_attn -- FlashAttention forward pass for NVIDIA B200 (sm_100a) with the paper's
+ * Sawtooth Wavefront Reordering of the K/V scan.  C ABI; no C++ types or exceptions cross it.
+ *
+ * What is computed (Eq. 1 of the paper; `scale` is the factor Algorithm 1 multiplies S by, 1/sqrt(d)
+ * in Eq. 1): for every batch b, head h and query row i,
+ *
+ *     O[b,h,i,:] = sum_j softmax_j( scale * Q[b,h,i,:] . K[b,h,j,:] ) * V[b,h,j,:]
+ *
+ * over the keys j the row may see: all N of them, or, under the causal mask, j <= i.
+ *
+ * How (Algorithms 1, 2 and 4): a persistent grid of G = min(#work items, #SMs) CTAs walks the work
+ * items k = blockIdx.x, += G; an item is a block of W query rows of one (b, h) that stays resident in
+ * shared memory while the K/V tiles of that head are streamed past it, with an online softmax.  In
+ * the cyclic order every item scans its K/V tiles first to last; in the sawtooth order a CTA scans
+ * first to last on its even iterations and last to first on its odd ones, so that the tiles it
+ * touched last are the ones it, and the CTAs running beside it, touch next, while they are still
+ * in L2.  Both orders give the same result up to the rounding order of the running sums.
+ *
+ * Layout: q, k, v, o are contiguous row-major [B, H, N, d] arrays (d fastest) of 16-bit elements,
+ * all of the same type (IEEE fp16 or bfloat16); N_q = N_k = N.  Products accumulate in fp32; the
+ * probabilities are rounded to the 16-bit type before the second product; O is rounded once at the
+ * end.  Supported: d in {64, 128}; any B, H, N >= 1 with B*H <= 2^31-1 and N <= 2^24; scale finite
+ * and > 0.  Every base pointer must be 16-byte aligned.  `o` must not overlap q, k or v.
+ *
+ * Ownership: the caller owns every buffer; the library allocates no device memory.  Calls enqueue
+ * work on the given stream and return without waiting (except where stated).  For fixed arguments
+ * the output is bitwise reproducible.
+ *
+ * Errors: every function that returns int returns ATTN_OK (0) or a negative attn_status;
+ * attn_last_error() then holds a description (per host thread).
+ */
+#ifndef SAWTOOTH_ATTN_H
+#define SAWTOOTH_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ATTN_OK = 0,
+    ATTN_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, unknown enum, bad scale, bad option */
+    ATTN_ERR_UNSUPPORTED = -2,    /* head dimension other than 64 / 128; device is not compute capability 10.x */
+    ATTN_ERR_ALIGNMENT = -3,      /* a base pointer is not 16-byte aligned */
+    ATTN_ERR_NO_DEVICE = -4,      /* no usable CUDA device / driver */
+    ATTN_ERR_CUDA = -5,           /* a CUDA runtime or driver call failed */
+    ATTN_ERR_DEVICE_TIMEOUT = -6  /* a bounded wait inside the kernel ran out (see attn_device_status) */
+} attn_status;
+
+typedef enum { ATTN_SCAN_CYCLIC = 0, ATTN_SCAN_SAWTOOTH = 1 } attn_scan_order;
+typedef enum { ATTN_F16 = 0, ATTN_BF16 = 1 } attn_dtype;
+typedef enum { ATTN_TILE_FASTEST = 0, ATTN_HEAD_FASTEST = 1 } attn_digit_order;
+
+/* Optional knobs; zero-initialise, then set what you need.  0 always means "library default". */
+typedef struct {
+    int max_ctas;     /* cap on the persistent grid (the "number of active SMs" of the paper's studies) */
+    int kv_stages;    /* K/V tile slots in the shared-memory ring; default: as many as fit */
+    int block_n;      /* K/V rows per tile: 64 or 128 (default 128) */
+    int q_tiles;      /* 128-row Q tiles per work item: 1 or 2 (default 2, so W = 256 rows) */
+    int digit_order;  /* attn_digit_order: how the linear work index maps to (batch, head, Q block) */
+    int launch_mode;  /* 0: persistent grid (Algorithm 2); 1: one CTA per work item (Algorithm 3) */
+    int l2_policy;    /* 0: no hint; 1: K/V loads carry an evict_last hint, Q loads evict_first */
+    int reserved[9];
+} attn_fwd_opts;
+
+/* What a call with these arguments will launch; lets a caller predict L2 traffic. */
+typedef struct {
+    int block_m;        /* query rows per MMA tile (128) */
+    int block_n;        /* K/V rows per tile */
+    int q_tiles;        /* Q tiles per work item */
+    int rows_per_item;  /* W = block_m * q_tiles */
+    int items_per_head; /* ceil(N / W) */
+    long long n_work;   /* B * H * items_per_head */
+    int grid;           /* CTAs launched */
+    int threads;        /* threads per CTA */
+    int kv_stages;      /* ring slots (each holds one K tile or one V tile) */
+    int smem_bytes;     /* dynamic shared memory per CTA */
+    int sm_count;       /* SMs of the device the plan was made for */
+} attn_plan;
+
+/* One work item as a CTA handles it (host-side replay of the device schedule). */
+typedef struct {
+    int cta;            /* blockIdx.x */
+    int iteration;      /* the CTA's local iteration count (Algorithm 4's i_local) */
+    long long k;        /* linear work index */
+    int batch, head;
+    int q_item;         /* index of the W-row block inside the head */
+    int backward;       /* 1: K/V tiles scanned last to first */
+    int n_kv;           /* tiles 0 .. n_kv-1 are scanned */
+    int n_kv_q0, n_kv_q1; /* of those, the ones the first / second 128-row Q tile takes part in */
+} attn_trace_entry;
+
+/*
+ * The forward pass (Eq. 1 via Algorithms 1, 2, 4).  q, k, v, o: DEVICE pointers, layout as above.
+ * causal: 0 or 1.  scan_order: attn_scan_order.  dtype: attn_dtype.  stream: a cudaStream_t (NULL =
+ * the default stream).  Asynchronous.  `o` is fully overwritten.
+ */
+int attn_fwd(const void* q, const void* k, const void* v, void* o,
+             int B, int H, int N, int d, float scale, int causal, int scan_order,
+             int dtype, void* stream);
+
+/* Same with options (opts may be NULL). */
+int attn_fwd_ex(const void* q, const void* k, const void* v, void* o,
+                int B, int H, int N, int d, float scale, int causal, int scan_order,
+                int dtype, void* stream, const attn_fwd_opts* opts);
+
+/*
+ * Same computation for HOST buffers: copies q, k, v (host, ideally pinned) into the caller's device
+ * staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host,
+ * all enqueued on `stream`.  Each buffer holds B*H*N*d 16-bit elements.  Returns without waiting:
+ * o_host is valid once the stream has been synchronised.
+ */
+int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                  void* q_dev, void* k_dev, void* v_dev, void* o_dev,
+                  int B, int H, int N, int d, float scale, int causal, int scan_order,
+                  int dtype, void* stream, const attn_fwd_opts* opts);
+
+/*
+ * The launch plan for these arguments (Algorithm 2's grid size, the tile shapes).  sm_count <= 0
+ * means "ask the current device" (fails with ATTN_ERR_NO_DEVICE without one).
+ */
+int attn_query_plan(int B, int H, int N, int d, int causal, int dtype,
+                    const attn_fwd_opts* opts, int sm_count, attn_plan* out);
+
+/*
+ * Host-only replay of the schedule (Algorithms 2 and 4 plus the causal tile ranges): writes up to
+ * `cap` entries, CTA by CTA, each CTA's items in the order it handles them, and the total number of
+ * entries to *n.  Needs no device when sm_count > 0.
+ */
+int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, int dtype,
+                        const attn_fwd_opts* opts, int sm_count,
+                        attn_trace_entry* buf, size_t cap, size_t* n);
+
+/*
+ * Waits for the current device and reads, then clears, its kernel status word: 0, or a code naming
+ * the wait that ran out in a kernel launched since the last call.  Returns ATTN_OK when the word
+ * was 0, ATTN_ERR_DEVICE_TIMEOUT otherwise (code in *code if code != NULL).
+ */
+int attn_device_status(int* code);
+
+const char* attn_status_string(int status);
+const char* attn_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAWTOOTH_ATTN_H */

@@ -1,0 +1,332 @@
+// C-ABI entry points of libsawtooth_attn: argument validation, launch plan, tensor maps, launch.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/sawtooth_attn.h"
+#include "attn_fwd_sm100.cuh"
+
+namespace {
+
+using namespace sawtooth;
+
+thread_local char g_error[512] = "";
+
+int fail(int status, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+__device__ int g_status_word = 0;
+
+constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
+
+struct Resolved {
+    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas;
+    size_t smem;
+};
+
+size_t smem_for(int d, int block_n, int q_tiles, int stages) {
+    return 1024 + (size_t)q_tiles * kBlockM * d * 2 + (size_t)stages * block_n * d * 2 + sizeof(Barriers);
+}
+
+int check_shape(int B, int H, int N, int d, int causal, int dtype) {
+    if (B <= 0 || H <= 0 || N <= 0) return fail(ATTN_ERR_INVALID_ARG, "B, H and N must be positive (got %d, %d, %d)", B, H, N);
+    if ((long long)B * H > 2147483647LL) return fail(ATTN_ERR_INVALID_ARG, "B*H exceeds 2^31-1");
+    if (N > (1 << 24)) return fail(ATTN_ERR_INVALID_ARG, "N exceeds 2^24");
+    if (d != 64 && d != 128) return fail(ATTN_ERR_UNSUPPORTED, "head dimension %d is not supported (64 or 128)", d);
+    if (causal != 0 && causal != 1) return fail(ATTN_ERR_INVALID_ARG, "causal must be 0 or 1");
+    if (dtype != ATTN_F16 && dtype != ATTN_BF16) return fail(ATTN_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    return ATTN_OK;
+}
+
+int resolve_opts(const attn_fwd_opts* o, int d, int smem_limit, Resolved* r) {
+    attn_fwd_opts z;
+    memset(&z, 0, sizeof(z));
+    if (o) z = *o;
+    r->block_n = z.block_n ? z.block_n : 128;
+    r->q_tiles = z.q_tiles ? z.q_tiles : 2;
+    if (r->block_n != 64 && r->block_n != 128) return fail(ATTN_ERR_INVALID_ARG, "block_n must be 64 or 128");
+    if (r->q_tiles != 1 && r->q_tiles != 2) return fail(ATTN_ERR_INVALID_ARG, "q_tiles must be 1 or 2");
+    if (z.digit_order != ATTN_TILE_FASTEST && z.digit_order != ATTN_HEAD_FASTEST)
+        return fail(ATTN_ERR_INVALID_ARG, "unknown digit_order %d", z.digit_order);
+    if (z.launch_mode != 0 && z.launch_mode != 1) return fail(ATTN_ERR_INVALID_ARG, "launch_mode must be 0 or 1");
+    if (z.l2_policy != 0 && z.l2_policy != 1) return fail(ATTN_ERR_INVALID_ARG, "l2_policy must be 0 or 1");
+    if (z.max_ctas < 0 || z.kv_stages < 0) return fail(ATTN_ERR_INVALID_ARG, "max_ctas and kv_stages must be >= 0");
+    r->head_fastest = z.digit_order == ATTN_HEAD_FASTEST;
+    r->launch_mode = z.launch_mode;
+    r->l2_policy = z.l2_policy;
+    r->max_ctas = z.max_ctas;
+    int fit = 0;
+    for (int s = kMaxStages; s >= 2; --s)
+        if (smem_for(d, r->block_n, r->q_tiles, s) <= (size_t)smem_limit) { fit = s; break; }
+    if (fit == 0) return fail(ATTN_ERR_UNSUPPORTED, "tile configuration does not fit in shared memory");
+    if (z.kv_stages) {
+        if (z.kv_stages < 2 || z.kv_stages > fit)
+            return fail(ATTN_ERR_INVALID_ARG, "kv_stages must be in [2, %d] for this configuration", fit);
+        fit = z.kv_stages;
+    }
+    r->stages = fit;
+    r->smem = smem_for(d, r->block_n, r->q_tiles, fit);
+    return ATTN_OK;
+}
+
+int device_sm_count(int* sms, int* smem_optin) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
+    if (major != 10) return fail(ATTN_ERR_UNSUPPORTED, "device compute capability %d.x is not 10.x", major);
+    cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    return ATTN_OK;
+}
+
+int grid_for(long long n_work, int sm_count, const Resolved& r) {
+    long long cap = sm_count;
+    if (r.max_ctas > 0 && r.max_ctas < cap) cap = r.max_ctas;
+    if (r.launch_mode == 1) return (int)(n_work < 2147483647LL ? n_work : 2147483647LL);  // Algorithm 3
+    return (int)(n_work < cap ? n_work : cap);                                           // Algorithm 2
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int get_encoder(EncodeTiledFn* fn) {
+    static EncodeTiledFn cached = nullptr;
+    if (!cached) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+            cudaGetLastError();
+            return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        }
+        cached = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    *fn = cached;
+    return ATTN_OK;
+}
+
+// [B*H, N, d] view, box = 64 columns x `rows` rows of one head, 128-byte swizzle, zero fill outside.
+int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype) {
+    EncodeTiledFn enc;
+    int rc = get_encoder(&enc);
+    if (rc) return rc;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, dtype == ATTN_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+    return ATTN_OK;
+}
+
+template <int kD, int kBlockN, int kQTiles, int kBf16>
+int launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const KernelParams& kp, int grid,
+           size_t smem, cudaStream_t stream) {
+    auto kern = attn_fwd_kernel<kD, kBlockN, kQTiles, kBf16>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); }
+    kern<<<grid, Geometry<kD, kBlockN, kQTiles>::kThreads, smem, stream>>>(tq, tk, tv, kp);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+    return ATTN_OK;
+}
+
+template <int kD, int kBlockN, int kQTiles>
+int launch_dtype(int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const KernelParams& kp,
+                 int grid, size_t smem, cudaStream_t stream) {
+    return dtype == ATTN_BF16 ? launch<kD, kBlockN, kQTiles, 1>(tq, tk, tv, kp, grid, smem, stream)
+                              : launch<kD, kBlockN, kQTiles, 0>(tq, tk, tv, kp, grid, smem, stream);
+}
+
+template <int kD>
+int launch_tiles(int block_n, int q_tiles, int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                 const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
+    if (block_n == 128) {
+        return q_tiles == 2 ? launch_dtype<kD, 128, 2>(dtype, tq, tk, tv, kp, grid, smem, stream)
+                            : launch_dtype<kD, 128, 1>(dtype, tq, tk, tv, kp, grid, smem, stream);
+    }
+    return q_tiles == 2 ? launch_dtype<kD, 64, 2>(dtype, tq, tk, tv, kp, grid, smem, stream)
+                        : launch_dtype<kD, 64, 1>(dtype, tq, tk, tv, kp, grid, smem, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* attn_status_string(int status) {
+    switch (status) {
+        case ATTN_OK: return "ok";
+        case ATTN_ERR_INVALID_ARG: return "invalid argument";
+        case ATTN_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case ATTN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case ATTN_ERR_NO_DEVICE: return "no CUDA device";
+        case ATTN_ERR_CUDA: return "CUDA call failed";
+        case ATTN_ERR_DEVICE_TIMEOUT: return "a bounded wait inside the kernel ran out";
+        default: return "unknown status";
+    }
+}
+
+const char* attn_last_error(void) { return g_error; }
+
+int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const attn_fwd_opts* opts, int sm_count,
+                    attn_plan* out) {
+    if (!out) return fail(ATTN_ERR_INVALID_ARG, "out is null");
+    int rc = check_shape(B, H, N, d, causal, dtype);
+    if (rc) return rc;
+    int smem_limit = kSmemOptinB200;
+    if (sm_count <= 0) {
+        rc = device_sm_count(&sm_count, &smem_limit);
+        if (rc) return rc;
+    }
+    Resolved r;
+    rc = resolve_opts(opts, d, smem_limit, &r);
+    if (rc) return rc;
+    const SchedParams sp = make_sched(B, H, N, r.q_tiles, r.block_n, causal, 0, r.head_fastest);
+    out->block_m = kBlockM;
+    out->block_n = r.block_n;
+    out->q_tiles = r.q_tiles;
+    out->rows_per_item = kBlockM * r.q_tiles;
+    out->items_per_head = sp.n_q;
+    out->n_work = sp.n_work;
+    out->grid = grid_for(sp.n_work, sm_count, r);
+    out->threads = r.q_tiles * 128 + 64;
+    out->kv_stages = r.stages;
+    out->smem_bytes = (int)r.smem;
+    out->sm_count = sm_count;
+    return ATTN_OK;
+}
+
+int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, int dtype, const attn_fwd_opts* opts,
+                        int sm_count, attn_trace_entry* buf, size_t cap, size_t* n) {
+    if (!n) return fail(ATTN_ERR_INVALID_ARG, "n is null");
+    if (cap > 0 && !buf) return fail(ATTN_ERR_INVALID_ARG, "buf is null");
+    if (scan_order != ATTN_SCAN_CYCLIC && scan_order != ATTN_SCAN_SAWTOOTH)
+        return fail(ATTN_ERR_INVALID_ARG, "unknown scan_order %d", scan_order);
+    attn_plan plan;
+    int rc = attn_query_plan(B, H, N, d, causal, dtype, opts, sm_count, &plan);
+    if (rc) return rc;
+    const int head_fastest = opts && opts->digit_order == ATTN_HEAD_FASTEST;
+    const SchedParams sp = make_sched(B, H, N, plan.q_tiles, plan.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, head_fastest);
+    size_t count = 0;
+    for (int cta = 0; cta < plan.grid; ++cta) {
+        int it = 0;
+        for (long long k = cta; k < sp.n_work; k += plan.grid, ++it) {
+            if (count < cap) {
+                const WorkItem w = decode_work(sp, k, it);
+                attn_trace_entry* e = &buf[count];
+                e->cta = cta;
+                e->iteration = it;
+                e->k = k;
+                e->batch = w.bh / H;
+                e->head = w.bh % H;
+                e->q_item = w.q_item;
+                e->backward = w.backward;
+                e->n_kv = w.hi;
+                e->n_kv_q0 = w.hi_q[0];
+                e->n_kv_q1 = w.hi_q[1];
+            }
+            ++count;
+        }
+    }
+    *n = count;
+    return ATTN_OK;
+}
+
+int attn_fwd_ex(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                int scan_order, int dtype, void* stream, const attn_fwd_opts* opts) {
+    if (!q || !k || !v || !o) return fail(ATTN_ERR_INVALID_ARG, "q, k, v and o must be non-null");
+    int rc = check_shape(B, H, N, d, causal, dtype);
+    if (rc) return rc;
+    if (scan_order != ATTN_SCAN_CYCLIC && scan_order != ATTN_SCAN_SAWTOOTH)
+        return fail(ATTN_ERR_INVALID_ARG, "unknown scan_order %d", scan_order);
+    if (!std::isfinite(scale) || !(scale > 0.f)) return fail(ATTN_ERR_INVALID_ARG, "scale must be finite and positive");
+    if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u)
+        return fail(ATTN_ERR_ALIGNMENT, "q, k, v and o must be 16-byte aligned");
+    int sm_count = 0, smem_limit = 0;
+    rc = device_sm_count(&sm_count, &smem_limit);
+    if (rc) return rc;
+    Resolved r;
+    rc = resolve_opts(opts, d, smem_limit, &r);
+    if (rc) return rc;
+
+    KernelParams kp;
+    kp.sched = make_sched(B, H, N, r.q_tiles, r.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, r.head_fastest);
+    kp.scale_log2 = scale * 1.4426950408889634f;
+    kp.kv_stages = r.stages;
+    kp.l2_policy = r.l2_policy;
+    kp.o = o;
+    rc = (int)cudaGetSymbolAddress((void**)&kp.status, g_status_word);
+    if (rc != 0) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress failed (%d)", rc); }
+
+    CUtensorMap tq, tk, tv;
+    if ((rc = make_map(&tq, q, B * H, N, d, kBlockM, dtype))) return rc;
+    if ((rc = make_map(&tk, k, B * H, N, d, r.block_n, dtype))) return rc;
+    if ((rc = make_map(&tv, v, B * H, N, d, r.block_n, dtype))) return rc;
+
+    const int grid = grid_for(kp.sched.n_work, sm_count, r);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st)
+                    : launch_tiles<64>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st);
+}
+
+int attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+             int scan_order, int dtype, void* stream) {
+    return attn_fwd_ex(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, nullptr);
+}
+
+int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, void* q_dev, void* k_dev,
+                  void* v_dev, void* o_dev, int B, int H, int N, int d, float scale, int causal, int scan_order, int dtype,
+                  void* stream, const attn_fwd_opts* opts) {
+    if (!q_host || !k_host || !v_host || !o_host) return fail(ATTN_ERR_INVALID_ARG, "host buffers must be non-null");
+    if (!q_dev || !k_dev || !v_dev || !o_dev) return fail(ATTN_ERR_INVALID_ARG, "device staging buffers must be non-null");
+    int rc = check_shape(B, H, N, d, causal, dtype);
+    if (rc) return rc;
+    const size_t bytes = (size_t)B * H * N * d * 2;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(v_dev, v_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ATTN_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
+    }
+    rc = attn_fwd_ex(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, stream, opts);
+    if (rc) return rc;
+    if ((e = cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ATTN_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
+    }
+    return ATTN_OK;
+}
+
+int attn_device_status(int* code) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e)); }
+    int word = 0;
+    e = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int));
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "reading the status word: %s", cudaGetErrorString(e)); }
+    if (code) *code = word;
+    if (word != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int));
+        return fail(ATTN_ERR_DEVICE_TIMEOUT, "kernel wait site %d ran out of time", word);
+    }
+    return ATTN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,415 @@
+// FlashAttention forward kernel for sm_100a: persistent CTAs, TMA-fed K/V ring, tcgen05 MMAs with
+// S, P and O in tensor memory, one softmax thread per query row.
+//
+// One CTA handles work items of kQTiles x 128 query rows (Algorithm 1's resident Q tile).  Warp roles:
+//   warps [0, 4*kQTiles)   softmax: warpgroup q owns the 128 rows of Q tile q, thread r owns row r
+//                          (TMEM lane r): reads S from TMEM, keeps the running max and sum, writes
+//                          P back to TMEM as 16-bit pairs, rescales O when the max moved, and at the
+//                          end of the item normalises O and stores it.
+//   warp 4*kQTiles         producer: one lane issues the TMA loads (Q tiles, then K_j, V_j in the
+//                          scan order of the item) into a ring of shared-memory slots.
+//   warp 4*kQTiles + 1     MMA: one lane issues S_q = Q_q K_j^T and O_q += P_q V_j and commits them
+//                          to mbarriers; the warp also owns the TMEM allocation.
+// With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
+#pragma once
+#include "ptx.cuh"
+#include "schedule.h"
+
+namespace sawtooth {
+
+struct KernelParams {
+    SchedParams sched;
+    float scale_log2;     // scale * log2(e): probabilities are computed with ex2
+    int kv_stages;        // slots in the K/V ring
+    int l2_policy;        // 1: K/V loads evict_last, Q loads evict_first
+    void* o;              // [B, H, N, d] output
+    int* status;          // device status word (0 = fine)
+};
+
+constexpr int kMaxStages = 16;
+constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the row max grew by more (log2 units)
+
+// Codes written to the status word: which wait gave up.
+enum WaitSite {
+    kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
+    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7
+};
+
+struct __align__(8) Barriers {
+    uint64_t q_full, q_empty;
+    uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int kD, int kBlockN, int kQTiles>
+struct Geometry {
+    static constexpr int kChunks = kD / 64;                 // 64-element (128-byte) column blocks per row
+    static constexpr int kQTileBytes = kBlockM * kD * 2;
+    static constexpr int kKVTileBytes = kBlockN * kD * 2;
+    static constexpr int kQChunkBytes = kBlockM * 128;
+    static constexpr int kKVChunkBytes = kBlockN * 128;
+    static constexpr int kSoftmaxThreads = kQTiles * 128;
+    static constexpr int kThreads = kSoftmaxThreads + 64;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q aliases its first kBlockN/2 columns
+    static constexpr int kTmemO = 256;    // O_q (fp32, kD columns) at kTmemO + 128 q
+    static constexpr size_t smem_bytes(int stages) {
+        return 1024 + (size_t)kQTiles * kQTileBytes + (size_t)stages * kKVTileBytes + sizeof(Barriers);
+    }
+};
+
+struct Ring {
+    int slot = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int stages) {
+        if (++slot == stages) { slot = 0; phase ^= 1u; }
+    }
+};
+
+// Short wait that ignores the abort flag: used on the way out, for copies and MMAs still in flight.
+__device__ __forceinline__ void drain_wait(uint64_t* bar, uint32_t parity) {
+    const unsigned long long t0 = ptx::global_ns();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (ptx::global_ns() - t0 > 2000000ull) break;
+    }
+}
+
+template <int kD, int kBlockN, int kQTiles, int kBf16>
+__global__ void __launch_bounds__(Geometry<kD, kBlockN, kQTiles>::kThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const KernelParams p)
+{
+    using G = Geometry<kD, kBlockN, kQTiles>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* q_smem = smem;
+    uint8_t* kv_smem = smem + kQTiles * G::kQTileBytes;
+    Barriers* bar = reinterpret_cast<Barriers*>(kv_smem + (size_t)p.kv_stages * G::kKVTileBytes);
+    volatile int* abort_flag = &bar->abort_flag;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    constexpr int kProducerWarp = 4 * kQTiles;
+    constexpr int kMmaWarp = 4 * kQTiles + 1;
+    const int stages = p.kv_stages;
+
+    if (tid == 0) {
+        ptx::mbar_init(&bar->q_full, 1);
+        ptx::mbar_init(&bar->q_empty, 1);
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(&bar->kv_full[s], 1);
+            ptx::mbar_init(&bar->kv_empty[s], 1);
+        }
+        for (int q = 0; q < 2; ++q) {
+            ptx::mbar_init(&bar->s_full[q], 1);
+            ptx::mbar_init(&bar->p_full[q], 128);
+            ptx::mbar_init(&bar->o_full[q], 1);
+        }
+        ptx::mbar_init(&bar->drain, 1);
+        bar->abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        ptx::prefetch_tmap(&tm_q);
+        ptx::prefetch_tmap(&tm_k);
+        ptx::prefetch_tmap(&tm_v);
+    }
+    if (warp == kMmaWarp) {
+        ptx::tmem_alloc(&bar->tmem_base, G::kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = bar->tmem_base;
+
+    const long long k_first = blockIdx.x;
+    const long long k_stride = gridDim.x;
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint64_t pol_kv = 0, pol_q = 0;
+            if (p.l2_policy) { pol_kv = ptx::policy_evict_last(); pol_q = ptx::policy_evict_first(); }
+            Ring ring;
+            uint32_t q_issued = 0;     // Q loads issued so far
+            long long kv_issued = 0;   // K/V tile loads issued so far
+            bool ok = true;
+            int it = 0;
+            for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+                const WorkItem w = decode_work(p.sched, k, it);
+                if (!ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ)) { ok = false; break; }
+                int n_valid = 0;
+                for (int q = 0; q < kQTiles; ++q) n_valid += (w.hi_q[q] > 0);
+                ptx::mbar_arrive_expect_tx(&bar->q_full, (uint32_t)n_valid * G::kQTileBytes);
+                for (int q = 0; q < kQTiles; ++q) {
+                    if (w.hi_q[q] == 0) continue;
+                    for (int c = 0; c < G::kChunks; ++c) {
+                        void* dst = q_smem + q * G::kQTileBytes + c * G::kQChunkBytes;
+                        if (p.l2_policy) ptx::tma_load_3d_hint(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh, pol_q);
+                        else ptx::tma_load_3d(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh);
+                    }
+                }
+                ++q_issued;
+                for (int s = 0; ok && s < w.hi; ++s) {
+                    const int j = kv_tile_at(w, s);
+                    for (int kv = 0; kv < 2; ++kv) {
+                        if (!ptx::mbar_wait(&bar->kv_empty[ring.slot], ring.phase ^ 1u, abort_flag, kSiteProducerKV)) { ok = false; break; }
+                        ptx::mbar_arrive_expect_tx(&bar->kv_full[ring.slot], G::kKVTileBytes);
+                        const CUtensorMap* tm = kv ? &tm_v : &tm_k;
+                        for (int c = 0; c < G::kChunks; ++c) {
+                            void* dst = kv_smem + (size_t)ring.slot * G::kKVTileBytes + c * G::kKVChunkBytes;
+                            if (p.l2_policy) ptx::tma_load_3d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh, pol_kv);
+                            else ptx::tma_load_3d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh);
+                        }
+                        ring.advance(stages);
+                        ++kv_issued;
+                    }
+                }
+            }
+            if (!ok) {
+                // Leave no copy in flight: wait (briefly) for the loads issued last into each slot.
+                if (q_issued) drain_wait(&bar->q_full, (q_issued - 1) & 1u);
+                const int back = kv_issued < stages ? (int)kv_issued : stages;
+                Ring r = ring;
+                for (int n = 0; n < back; ++n) {
+                    if (r.slot == 0) { r.slot = stages - 1; r.phase ^= 1u; } else { --r.slot; }
+                    drain_wait(&bar->kv_full[r.slot], r.phase);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
+            constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
+            const uint32_t q_base = ptx::smem_u32(q_smem);
+            const uint32_t kv_base = ptx::smem_u32(kv_smem);
+            Ring ring;
+            uint32_t p_phase[2] = {0, 0};
+            bool ok = true;
+
+            auto issue_qk = [&](int q, int slot) {
+                const uint32_t a0 = q_base + q * G::kQTileBytes;
+                const uint32_t b0 = kv_base + slot * G::kKVTileBytes;
+#pragma unroll
+                for (int c = 0; c < G::kChunks; ++c) {
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t a = ptx::smem_desc_sw128(a0 + c * G::kQChunkBytes + kk * 32, 16, 1024);
+                        const uint64_t b = ptx::smem_desc_sw128(b0 + c * G::kKVChunkBytes + kk * 32, 16, 1024);
+                        ptx::mma_ss(tmem + G::kTmemS + 128 * q, a, b, idesc_qk, (c | kk) != 0);
+                    }
+                }
+            };
+            auto issue_pv = [&](int q, int slot, uint32_t accumulate) {
+                const uint32_t b0 = kv_base + slot * G::kKVTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < kBlockN / 16; ++kk) {
+                    const uint64_t b = ptx::smem_desc_sw128(b0 + kk * 16 * 128, G::kKVChunkBytes, 1024);
+                    ptx::mma_ts(tmem + G::kTmemO + 128 * q, tmem + G::kTmemS + 128 * q + kk * 8, b, idesc_pv,
+                                accumulate | (kk != 0));
+                }
+            };
+
+            int it = 0;
+            for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+                const WorkItem w = decode_work(p.sched, k, it);
+                if (!ptx::mbar_wait(&bar->q_full, it & 1, abort_flag, kSiteMmaQ)) { ok = false; break; }
+                // K tile of step 0
+                int slot_k = ring.slot;
+                if (!ptx::mbar_wait(&bar->kv_full[slot_k], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                ring.advance(stages);
+                ptx::tc_fence_after();
+                {
+                    const int j0 = kv_tile_at(w, 0);
+                    for (int q = 0; q < kQTiles; ++q) {
+                        if (j0 < w.hi_q[q]) { issue_qk(q, slot_k); ptx::mma_commit(&bar->s_full[q]); }
+                    }
+                    ptx::mma_commit(&bar->kv_empty[slot_k]);
+                    if (w.hi == 1) ptx::mma_commit(&bar->q_empty);
+                }
+                uint32_t pv_started[2] = {0, 0};
+                for (int s = 0; ok && s < w.hi; ++s) {
+                    const int j = kv_tile_at(w, s);
+                    const bool has_next = s + 1 < w.hi;
+                    const int j_next = has_next ? kv_tile_at(w, s + 1) : 0;
+                    const int slot_v = ring.slot;
+                    if (!ptx::mbar_wait(&bar->kv_full[slot_v], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                    ring.advance(stages);
+                    int slot_kn = 0;
+                    if (has_next) {
+                        slot_kn = ring.slot;
+                        if (!ptx::mbar_wait(&bar->kv_full[slot_kn], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                        ring.advance(stages);
+                    }
+                    for (int q = 0; q < kQTiles; ++q) {
+                        if (j < w.hi_q[q]) {
+                            if (!ptx::mbar_wait(&bar->p_full[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
+                            p_phase[q] ^= 1u;
+                            ptx::tc_fence_after();
+                            issue_pv(q, slot_v, pv_started[q]);
+                            pv_started[q] = 1;
+                        }
+                        if (has_next && j_next < w.hi_q[q]) {
+                            issue_qk(q, slot_kn);
+                            ptx::mma_commit(&bar->s_full[q]);
+                        }
+                    }
+                    if (!ok) break;
+                    ptx::mma_commit(&bar->kv_empty[slot_v]);
+                    if (has_next) {
+                        ptx::mma_commit(&bar->kv_empty[slot_kn]);
+                        if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S products are issued
+                    }
+                }
+                if (!ok) break;
+                for (int q = 0; q < kQTiles; ++q)
+                    if (w.hi_q[q] > 0) ptx::mma_commit(&bar->o_full[q]);
+            }
+            // Nothing of this thread's MMAs may be in flight when TMEM is released.
+            ptx::mma_commit(&bar->drain);
+            drain_wait(&bar->drain, 0);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ softmax / correction / epilogue
+        const int q = warp >> 2;                       // which Q tile this warpgroup owns
+        const int r_in_tile = tid & 127;               // row inside the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + G::kTmemS + 128 * q;
+        const uint32_t t_o = tmem + lane_base + G::kTmemO + 128 * q;
+        const float scale_log2 = p.scale_log2;
+        const int N = p.sched.N;
+        uint32_t s_phase = 0, o_phase = 0;
+        bool ok = true;
+        int it = 0;
+        for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+            const WorkItem w = decode_work(p.sched, k, it);
+            if (w.hi_q[q] == 0) continue;
+            const int tile_row0 = w.row0 + q * kBlockM;
+            const int row = tile_row0 + r_in_tile;
+            float m_ref = -INFINITY;   // the max the exponents are taken against (log2 units)
+            float l = 0.f;             // running sum of the probabilities
+            bool first = true;
+            for (int s = 0; s < w.hi; ++s) {
+                const int j = kv_tile_at(w, s);
+                if (j >= w.hi_q[q]) continue;
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS));
+                if (!ok) break;
+                s_phase ^= 1u;
+                ptx::tc_fence_after();
+
+                uint32_t sv[kBlockN / 32][32];
+#pragma unroll
+                for (int c = 0; c < kBlockN / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
+                ptx::tmem_wait_ld();
+
+                const int col0 = j * kBlockN;
+                const bool masked = (col0 + kBlockN > N) || (p.sched.causal && (col0 + kBlockN - 1 > tile_row0));
+                if (masked) {
+                    const int limit = p.sched.causal ? (row < N - 1 ? row : N - 1) : N - 1;  // last visible key
+#pragma unroll
+                    for (int c = 0; c < kBlockN / 32; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + c * 32 + i > limit) sv[c][i] = 0xff800000u;  // -inf
+                }
+
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < kBlockN / 32; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        mx0 = fmaxf(mx0, __uint_as_float(sv[c][i]));
+                        mx1 = fmaxf(mx1, __uint_as_float(sv[c][i + 1]));
+                        mx2 = fmaxf(mx2, __uint_as_float(sv[c][i + 2]));
+                        mx3 = fmaxf(mx3, __uint_as_float(sv[c][i + 3]));
+                    }
+                const float m_cand = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2);
+                const bool need = (m_cand - m_ref) > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    float alpha = 1.f;
+                    if (need) {
+                        alpha = ptx::ex2(m_ref - m_cand);  // 0 when nothing was accumulated yet
+                        m_ref = m_cand;
+                        l *= alpha;
+                    }
+                    if (!first) {
+                        // S_q is complete, so every product issued before it, O_q's last update included, is too.
+#pragma unroll
+                        for (int c = 0; c < kD / 32; ++c) {
+                            uint32_t ov[32];
+                            ptx::tmem_ld32(t_o + c * 32, ov);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                            ptx::tmem_st32(t_o + c * 32, ov);
+                        }
+                    }
+                }
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+                for (int c = 0; c < kBlockN / 32; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[c][i]), scale_log2, neg_m));
+                        const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 1]), scale_log2, neg_m));
+                        const float p2 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 2]), scale_log2, neg_m));
+                        const float p3 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 3]), scale_log2, neg_m));
+                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                        pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
+                        pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
+                    }
+                    ptx::tmem_st16(t_s + c * 16, pk);
+                }
+                l += (l0 + l1) + (l2 + l3);
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(&bar->p_full[q]);
+                first = false;
+            }
+            if (!ok) break;
+            // ---- epilogue: O_q / l -> 16 bit -> global
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bar->o_full[q], o_phase, abort_flag, kSiteSoftmaxO));
+            if (!ok) break;
+            o_phase ^= 1u;
+            ptx::tc_fence_after();
+            const float inv_l = 1.f / l;
+            uint4* o_row = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.o) + ((size_t)w.bh * N + row) * (size_t)(kD * 2));
+#pragma unroll
+            for (int c = 0; c < kD / 32; ++c) {
+                uint32_t ov[32];
+                ptx::tmem_ld32(t_o + c * 32, ov);
+                ptx::tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2)
+                    pk[i / 2] = ptx::pack2<kBf16>(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l);
+                if (row < N) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4)
+                        o_row[c * 4 + v4] = make_uint4(pk[4 * v4], pk[4 * v4 + 1], pk[4 * v4 + 2], pk[4 * v4 + 3]);
+                }
+            }
+            ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, G::kTmemCols);
+    }
+    if (tid == 0 && bar->abort_flag != 0) atomicCAS(p.status, 0, bar->abort_flag);
+}
+
+}  // namespace sawtooth

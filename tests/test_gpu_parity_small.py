@@ -1,0 +1,121 @@
+"""GPU parity at small and ragged sizes: every row of every head against the fp64 oracle, through
+the C ABI, for both scan orders, both tile shapes, one or two Q tiles per work item."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from parity_util import assert_parity, run_cuda, upload, output_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def opts_for(block_n=0, q_tiles=0, **kw):
+    import paper_2601_16032_b200 as sa
+    o = sa.Opts()
+    o.block_n, o.q_tiles = block_n, q_tiles
+    for k, v in kw.items():
+        setattr(o, k, v)
+    return o
+
+
+@pytest.mark.parametrize("N", [1, 17, 128, 129, 200, 256, 257, 1000])
+@pytest.mark.parametrize("d,dtype", [(64, wl.F16), (128, wl.BF16), (64, wl.BF16), (128, wl.F16)])
+@pytest.mark.parametrize("causal", [False, True])
+def test_ragged_sizes(N, d, dtype, causal):
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("ragged", 2, 3, N, d, dtype, causal, 7000 + N)
+    qkv = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        assert_parity(w, run_cuda(w, qkv, order))
+
+
+@pytest.mark.parametrize("block_n", [64, 128])
+@pytest.mark.parametrize("q_tiles", [1, 2])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("d,dtype", [(64, wl.F16), (128, wl.BF16)])
+def test_tile_shapes_and_scan_orders(block_n, q_tiles, causal, d, dtype):
+    """Few SMs' worth of CTAs (max_ctas) so that every CTA runs several items and alternates direction."""
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("tiles", 1, 2, 1330, d, dtype, causal, 7100 + block_n + q_tiles)
+    qkv = upload(w)
+    outs = []
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        o = run_cuda(w, qkv, order, opts_for(block_n, q_tiles, max_ctas=3))
+        assert_parity(w, o)
+        outs.append(o)
+    a = wl.bits_to_f64(output_bits(outs[0], 0, 1), dtype)
+    b = wl.bits_to_f64(output_bits(outs[1], 0, 1), dtype)
+    assert np.abs(a - b).max() <= 1e-2  # the two orders agree to rounding
+
+
+@pytest.mark.parametrize("opt", [dict(kv_stages=2), dict(kv_stages=3), dict(digit_order=1), dict(launch_mode=1),
+                                 dict(l2_policy=1), dict(max_ctas=1)])
+def test_options_do_not_change_the_result(opt):
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("opts", 2, 2, 900, 128, wl.BF16, True, 7200)
+    qkv = upload(w)
+    assert_parity(w, run_cuda(w, qkv, sa.SAWTOOTH, opts_for(**opt)))
+
+
+def test_bitwise_reproducible_and_guard_bands_untouched():
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("repro", 1, 2, 777, 128, wl.BF16, True, 7300)
+    q, k, v = upload(w)
+    n = q.numel()
+    guard = 4096
+    buf = torch.full((n + 2 * guard,), -1, dtype=torch.int16, device="cuda:0")
+    o = buf[guard:guard + n].view(torch.bfloat16).view(q.shape)
+    outs = []
+    for _ in range(2):
+        o.view(torch.int16).fill_(-1)
+        sa.attn_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, 1,
+                    sa.SAWTOOTH, sa.BF16, torch.cuda.current_stream().cuda_stream)
+        sa.attn_device_status()
+        outs.append(o.view(torch.int16).clone())
+        assert (buf[:guard] == -1).all() and (buf[guard + n:] == -1).all()
+    assert torch.equal(outs[0], outs[1])
+    assert_parity(w, o)
+
+
+def test_invariants_on_gpu():
+    """V = ones gives ones; causal row 0 returns V row 0; a dominant score selects its V row."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    B, H, N, d = 1, 2, 300, 64
+    g = torch.Generator(device="cpu").manual_seed(5)
+    q = torch.randn(B, H, N, d, generator=g).to(torch.float16).cuda()
+    k = torch.randn(B, H, N, d, generator=g).to(torch.float16).cuda()
+    v = torch.randn(B, H, N, d, generator=g).to(torch.float16).cuda()
+    ones = torch.ones_like(v)
+    for causal in (False, True):
+        o = sa.forward(q, k, ones, causal=causal)
+        sa.attn_device_status()
+        assert (o == 1).all()
+    o = sa.forward(q, k, v, causal=True)
+    sa.attn_device_status()
+    assert torch.equal(o[:, :, 0], v[:, :, 0])
+    kn = torch.nn.functional.normalize(k.float(), dim=-1)
+    q_hot = (60.0 * kn[:, :, 123:124]).expand(B, H, N, d).to(torch.float16).contiguous()
+    o = sa.forward(q_hot, kn.to(torch.float16), v, causal=False, scale=1.0)
+    sa.attn_device_status()
+    assert (o - v[:, :, 123:124]).abs().max() < 2e-2
+
+
+def test_bad_arguments_are_rejected_before_launch():
+    import torch
+    import paper_2601_16032_b200 as sa
+    t = torch.zeros(1, 1, 128, 64, dtype=torch.float16, device="cuda:0")
+    p = t.data_ptr()
+    st = 0
+    cases = [
+        (dict(q=0), -1), (dict(N=0), -1), (dict(d=96), -2), (dict(scale=float("nan")), -1), (dict(scale=-1.0), -1),
+        (dict(scan_order=5), -1), (dict(dtype=7), -1), (dict(causal=2), -1), (dict(q=p + 2), -3),
+    ]
+    for change, status in cases:
+        a = dict(q=p, k=p, v=p, o=p, B=1, H=1, N=128, d=64, scale=0.125, causal=0, scan_order=0, dtype=0)
+        a.update(change)
+        with pytest.raises(sa.AttnError) as e:
+            sa.attn_fwd(a["q"], a["k"], a["v"], a["o"], a["B"], a["H"], a["N"], a["d"], a["scale"], a["causal"],
+                        a["scan_order"], a["dtype"], st)
+        assert e.value.status == status, (change, e.value)
