@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the attention forward pass (one step = one attn_fwd call over the whole workload).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl reference]
+
+Prints ONE JSON line.  `value` is attention-forward TFLOP/s (4*B*H*N^2*d, halved under the causal
+mask) of the sawtooth scan order with the inputs resident in HBM; the cyclic order is timed the same
+way and reported beside it.  `e2e` goes through attn_fwd_host with pinned host buffers, copies
+included.  `roofline` compares the kernel with the measured bf16 tensor peak of this GPU pool,
+`cpu_baseline` times the fp64 oracle on a bounded sample of the same workload.
+
+With --gpus N > 1 (under torchrun) every rank runs the same workload on its own GPU: the path has no
+exchange step, so the ranks are independent replicas and `value` is the sum of their throughputs
+over the slowest rank's time.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import workloads as wl
+
+METRIC = "attention_fwd_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_BF16_TFLOPS = 1590.0
+# DRAM bytes one launch of the bench workload moves (dram__bytes_read.sum + dram__bytes_write.sum of
+# an ncu capture of the same kernel; see the summary under profiles/).  None until captured.
+NCU_DRAM_BYTES_PER_LAUNCH = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"burst": float(p["bf16_tflops"]), "sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    except Exception:
+        return {"burst": FALLBACK_BF16_TFLOPS, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_sample_heads(w: wl.Workload, n_heads: int):
+    return list(wl.all_heads(w))[:n_heads]
+
+
+def time_oracle(w: wl.Workload, heads, threads: int = 0):
+    """Seconds the oracle takes for every row of the given heads, and the FLOPs that is."""
+    from oracle import attention as ora
+    total, flops = 0.0, 0.0
+    for b, h in heads:
+        q = wl.bits_to_f64(wl.head_bits(w, "q", b, h), w.dtype)
+        k = wl.bits_to_f64(wl.head_bits(w, "k", b, h), w.dtype)
+        v = wl.bits_to_f64(wl.head_bits(w, "v", b, h), w.dtype)
+        idx = np.arange(w.N, dtype=np.int64)
+        t0 = time.perf_counter()
+        ora.attention_rows(q, idx, k, v, w.scale, w.causal, threads)
+        total += time.perf_counter() - t0
+        flops += 4.0 * float(w.N) ** 2 * w.d / (2 if w.causal else 1)
+    return total, flops
+
+
+def config_of(w: wl.Workload, extra=None):
+    c = {"workload": f"{w.name}: B={w.B} H={w.H} N={w.N} d={w.d} {w.dtype} {'causal' if w.causal else 'non-causal'}",
+         "seed": w.seed, "scale": "1/sqrt(d)", "k_scale": w.k_scale,
+         "l2": "inputs larger than L2 (Q+K+V+O = %d MiB)" % (w.compulsory_bytes >> 20)}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def run_reference(args, w: wl.Workload):
+    """The CPU oracle as the reference arm: each step computes every row of one head."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import attention as ora
+    heads = list(wl.all_heads(w))
+    for i in range(args.warmup):
+        time_oracle(w, [heads[i % len(heads)]])
+    secs, flops = 0.0, 0.0
+    for i in range(args.steps):
+        s, f = time_oracle(w, [heads[i % len(heads)]])
+        secs += s
+        flops += f
+    value = flops / secs / 1e12
+    sample = f"per step: every query row of one head of {w.name} ({w.N} rows x {w.N} keys, d={w.d})"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_of(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": ora.threads_available(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c3", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (default: min(steps, 10))")
+    ap.add_argument("--cpu-heads", type=int, default=-1, help="heads the CPU baseline computes (default: sized to ~15 s)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = wl.CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import paper_2601_16032_b200 as sa
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    dev = torch.device("cuda", local)
+    tdt = torch.bfloat16 if w.dtype == wl.BF16 else torch.float16
+    adt = sa.BF16 if w.dtype == wl.BF16 else sa.F16
+    shape = (w.B, w.H, w.N, w.d)
+    numel = w.B * w.H * w.N * w.d
+
+    # Inputs: the seeded workload, generated on the host into pinned buffers (they also feed the e2e leg).
+    host = {}
+    for name in ("q", "k", "v"):
+        t = torch.empty(shape, dtype=torch.int16).pin_memory()
+        arr = t.numpy()
+        for b, h in wl.all_heads(w):
+            arr[b, h] = wl.head_bits(w, name, b, h).view(np.int16)
+        host[name] = t
+    host["o"] = torch.empty(shape, dtype=torch.int16).pin_memory()
+    devb = {n: torch.empty(shape, dtype=torch.int16, device=dev) for n in ("q", "k", "v", "o")}
+    for n in ("q", "k", "v"):
+        devb[n].copy_(host[n])
+    stream = torch.cuda.Stream(device=dev)
+    sh = stream.cuda_stream
+
+    def step(order):
+        sa.attn_fwd(devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
+                    w.B, w.H, w.N, w.d, w.scale, int(w.causal), order, adt, sh)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                fn()
+            e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    results = {}
+    with ClockSampler(local) as clocks:
+        for order, name in ((sa.CYCLIC, "cyclic"), (sa.SAWTOOTH, "sawtooth")):
+            for _ in range(args.warmup):
+                step(order)
+            ms = timed(lambda: step(order), args.steps)
+            results[name] = ms / args.steps
+    sa.attn_device_status()
+    clk = clocks.summary()
+
+    # End to end: host buffers in, host buffer out, copies inside the timed region.
+    e2e_steps = args.e2e_steps or min(args.steps, 10)
+
+    def e2e_step():
+        sa.attn_fwd_host(host["q"].data_ptr(), host["k"].data_ptr(), host["v"].data_ptr(), host["o"].data_ptr(),
+                         devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
+                         w.B, w.H, w.N, w.d, w.scale, int(w.causal), sa.SAWTOOTH, adt, sh)
+
+    for _ in range(2):
+        e2e_step()
+    e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
+    sa.attn_device_status()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops = w.flops
+    ms_saw, ms_cyc = results["sawtooth"], results["cyclic"]
+    tf_saw = flops / ms_saw / 1e9
+    tf_cyc = flops / ms_cyc / 1e9
+    timed_region_s = ms_saw * args.steps / 1e3
+    peak_kind = "sustained" if timed_region_s >= 0.5 else "burst"
+    peak = peaks[peak_kind]
+    plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt)
+    line = {
+        "metric": METRIC, "value": tf_saw * world, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_saw, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == wl.BF16 else "f16", "data": "synthetic",
+        "config": config_of(w, {"scan_order": "sawtooth", "parallelism": "replicas only" if world > 1 else "single GPU",
+                                "grid": plan.grid, "rows_per_item": plan.rows_per_item, "block_n": plan.block_n,
+                                "kv_stages": plan.kv_stages}),
+        "cyclic": {"value": tf_cyc * world, "unit": UNIT, "ms_per_step": ms_cyc},
+        "sawtooth_over_cyclic": tf_saw / tf_cyc,
+        "clocks": clk,
+        "e2e": {"value": flops / e2e_ms / 1e9 * world, "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                "h2d_bytes_per_step": 3 * numel * 2, "d2h_bytes_per_step": numel * 2},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "tensor", "achieved": tf_saw, "peak": peak, "unit": UNIT, "frac": tf_saw / peak,
+                     "peak_kind": f"{peak_kind} bf16 matmul, of {peaks['source']}",
+                     "frac_of_burst": tf_saw / peaks["burst"], "frac_of_sustained": tf_saw / peaks["sustained"],
+                     "frac_of_nominal_2250": tf_saw / NOMINAL_BF16_TFLOPS,
+                     "flops_per_launch": flops, "launch_ms": ms_saw,
+                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name), "compulsory_bytes": w.compulsory_bytes},
+    }
+    if not args.skip_cpu_baseline:
+        from oracle import attention as ora
+        per_head_flops = 4.0 * float(w.N) ** 2 * w.d / (2 if w.causal else 1)
+        n_heads = args.cpu_heads if args.cpu_heads > 0 else max(1, min(w.B * w.H, int(15.0 * 2.5e9 * ora.threads_available() / per_head_flops)))
+        heads = oracle_sample_heads(w, n_heads)
+        secs, fl = time_oracle(w, heads)
+        line["cpu_baseline"] = {"value": fl / secs / 1e12, "unit": UNIT, "cores": ora.threads_available(), "kind": "oracle",
+                                "seconds": secs,
+                                "sample": f"every query row of the first {len(heads)} of {w.B * w.H} heads of {w.name}"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

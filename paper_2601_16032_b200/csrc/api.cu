@@ -204,7 +204,7 @@ int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const att
     out->items_per_head = sp.n_q;
     out->n_work = sp.n_work;
     out->grid = grid_for(sp.n_work, sm_count, r);
-    out->threads = r.q_tiles * 128 + 64;
+    out->threads = r.q_tiles * 128 + 128;
     out->kv_stages = r.stages;
     out->smem_bytes = (int)r.smem;
     out->sm_count = sm_count;

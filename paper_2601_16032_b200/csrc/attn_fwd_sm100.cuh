@@ -10,6 +10,7 @@
 //                          scan order of the item) into a ring of shared-memory slots.
 //   warp 4*kQTiles + 1     MMA: one lane issues S_q = Q_q K_j^T and O_q += P_q V_j and commits them
 //                          to mbarriers; the warp also owns the TMEM allocation.
+//   two more warps         idle; they complete the warpgroup whose registers go to the softmax threads.
 // With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
 #pragma once
 #include "ptx.cuh"
@@ -52,7 +53,13 @@ struct Geometry {
     static constexpr int kQChunkBytes = kBlockM * 128;
     static constexpr int kKVChunkBytes = kBlockN * 128;
     static constexpr int kSoftmaxThreads = kQTiles * 128;
-    static constexpr int kThreads = kSoftmaxThreads + 64;
+    static constexpr int kThreads = kSoftmaxThreads + 128;  // a full fourth/third warpgroup: producer, MMA, two idle warps
+    // Registers: the launch gives every thread 65536 / kThreads (rounded down to a multiple of 8).  With
+    // two Q tiles that is 168, too few for a softmax thread holding a 128-wide score row, so the last
+    // warpgroup hands registers back and the softmax warpgroups take them.
+    static constexpr bool kRebalance = (kQTiles == 2);
+    static constexpr int kRegsOther = 104;
+    static constexpr int kRegsSoftmax = 200;
     static constexpr int kTmemCols = 512;
     static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q aliases its first kBlockN/2 columns
     static constexpr int kTmemO = 256;    // O_q (fp32, kD columns) at kTmemO + 128 q
@@ -132,6 +139,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
+        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
         if (lane == 0) {
             uint64_t pol_kv = 0, pol_q = 0;
             if (p.l2_policy) { pol_kv = ptx::policy_evict_last(); pol_q = ptx::policy_evict_first(); }
@@ -144,10 +152,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const WorkItem w = decode_work(p.sched, k, it);
                 if (!ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ)) { ok = false; break; }
                 int n_valid = 0;
+#pragma unroll
                 for (int q = 0; q < kQTiles; ++q) n_valid += (w.hi_q[q] > 0);
                 ptx::mbar_arrive_expect_tx(&bar->q_full, (uint32_t)n_valid * G::kQTileBytes);
+#pragma unroll
                 for (int q = 0; q < kQTiles; ++q) {
                     if (w.hi_q[q] == 0) continue;
+#pragma unroll
                     for (int c = 0; c < G::kChunks; ++c) {
                         void* dst = q_smem + q * G::kQTileBytes + c * G::kQChunkBytes;
                         if (p.l2_policy) ptx::tma_load_3d_hint(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh, pol_q);
@@ -185,6 +196,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue
+        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
         if (lane == 0) {
             constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
             constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
@@ -194,25 +206,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             uint32_t p_phase[2] = {0, 0};
             bool ok = true;
 
+            // Descriptors differ from a base only in the 16-byte-granular address field (the low bits).
+            const uint64_t q_desc0 = ptx::smem_desc_sw128(q_base, 16, 1024);
+            const uint64_t k_desc0 = ptx::smem_desc_sw128(kv_base, 16, 1024);
+            const uint64_t v_desc0 = ptx::smem_desc_sw128(kv_base, G::kKVChunkBytes, 1024);
             auto issue_qk = [&](int q, int slot) {
-                const uint32_t a0 = q_base + q * G::kQTileBytes;
-                const uint32_t b0 = kv_base + slot * G::kKVTileBytes;
+                const uint64_t a0 = q_desc0 + (uint64_t)((q * G::kQTileBytes) >> 4);
+                const uint64_t b0 = k_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
+                const uint32_t d_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
-                for (int c = 0; c < G::kChunks; ++c) {
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t a = ptx::smem_desc_sw128(a0 + c * G::kQChunkBytes + kk * 32, 16, 1024);
-                        const uint64_t b = ptx::smem_desc_sw128(b0 + c * G::kKVChunkBytes + kk * 32, 16, 1024);
-                        ptx::mma_ss(tmem + G::kTmemS + 128 * q, a, b, idesc_qk, (c | kk) != 0);
-                    }
+                for (int i = 0; i < G::kChunks * 4; ++i) {
+                    const int c = i >> 2, kk = i & 3;
+                    ptx::mma_ss(d_tmem, a0 + (uint64_t)((c * G::kQChunkBytes + kk * 32) >> 4),
+                                b0 + (uint64_t)((c * G::kKVChunkBytes + kk * 32) >> 4), idesc_qk, i != 0);
                 }
             };
             auto issue_pv = [&](int q, int slot, uint32_t accumulate) {
-                const uint32_t b0 = kv_base + slot * G::kKVTileBytes;
+                const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
+                const uint32_t d_tmem = tmem + G::kTmemO + 128 * q;
+                const uint32_t a_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
                 for (int kk = 0; kk < kBlockN / 16; ++kk) {
-                    const uint64_t b = ptx::smem_desc_sw128(b0 + kk * 16 * 128, G::kKVChunkBytes, 1024);
-                    ptx::mma_ts(tmem + G::kTmemO + 128 * q, tmem + G::kTmemS + 128 * q + kk * 8, b, idesc_pv,
+                    ptx::mma_ts(d_tmem, a_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
                                 accumulate | (kk != 0));
                 }
             };
@@ -228,6 +243,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ptx::tc_fence_after();
                 {
                     const int j0 = kv_tile_at(w, 0);
+#pragma unroll
                     for (int q = 0; q < kQTiles; ++q) {
                         if (j0 < w.hi_q[q]) { issue_qk(q, slot_k); ptx::mma_commit(&bar->s_full[q]); }
                     }
@@ -248,6 +264,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (!ptx::mbar_wait(&bar->kv_full[slot_kn], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                         ring.advance(stages);
                     }
+#pragma unroll
                     for (int q = 0; q < kQTiles; ++q) {
                         if (j < w.hi_q[q]) {
                             if (!ptx::mbar_wait(&bar->p_full[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
@@ -269,6 +286,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 if (!ok) break;
+#pragma unroll
                 for (int q = 0; q < kQTiles; ++q)
                     if (w.hi_q[q] > 0) ptx::mma_commit(&bar->o_full[q]);
             }
@@ -277,8 +295,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             drain_wait(&bar->drain, 0);
         }
         __syncwarp();
-    } else {
+    } else if (warp < 4 * kQTiles) {
         // ------------------------------------------------------------------ softmax / correction / epilogue
+        if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
         const int q = warp >> 2;                       // which Q tile this warpgroup owns
         const int r_in_tile = tid & 127;               // row inside the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -291,7 +310,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         int it = 0;
         for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
             const WorkItem w = decode_work(p.sched, k, it);
-            if (w.hi_q[q] == 0) continue;
+            const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
+            if (hi_mine == 0) continue;
             const int tile_row0 = w.row0 + q * kBlockM;
             const int row = tile_row0 + r_in_tile;
             float m_ref = -INFINITY;   // the max the exponents are taken against (log2 units)
@@ -299,7 +319,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool first = true;
             for (int s = 0; s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
-                if (j >= w.hi_q[q]) continue;
+                if (j >= hi_mine) continue;
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS));
                 if (!ok) break;
                 s_phase ^= 1u;
@@ -325,11 +345,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int c = 0; c < kBlockN / 32; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        mx0 = fmaxf(mx0, __uint_as_float(sv[c][i]));
-                        mx1 = fmaxf(mx1, __uint_as_float(sv[c][i + 1]));
-                        mx2 = fmaxf(mx2, __uint_as_float(sv[c][i + 2]));
-                        mx3 = fmaxf(mx3, __uint_as_float(sv[c][i + 3]));
+                    for (int i = 0; i < 32; i += 8) {
+                        mx0 = ptx::max3(mx0, __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
+                        mx1 = ptx::max3(mx1, __uint_as_float(sv[c][i + 2]), __uint_as_float(sv[c][i + 3]));
+                        mx2 = ptx::max3(mx2, __uint_as_float(sv[c][i + 4]), __uint_as_float(sv[c][i + 5]));
+                        mx3 = ptx::max3(mx3, __uint_as_float(sv[c][i + 6]), __uint_as_float(sv[c][i + 7]));
                     }
                 const float m_cand = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2);
                 const bool need = (m_cand - m_ref) > kRescaleThreshold;
@@ -342,14 +362,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                     if (!first) {
                         // S_q is complete, so every product issued before it, O_q's last update included, is too.
-#pragma unroll
-                        for (int c = 0; c < kD / 32; ++c) {
-                            uint32_t ov[32];
-                            ptx::tmem_ld32(t_o + c * 32, ov);
+#pragma unroll 1
+                        for (int c = 0; c < kD / 16; ++c) {
+                            uint32_t ov[16];
+                            ptx::tmem_ld16(t_o + c * 16, ov);
                             ptx::tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                            ptx::tmem_st32(t_o + c * 32, ov);
+                            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                            ptx::tmem_st16(t_o + c * 16, ov);
                         }
                     }
                 }
@@ -357,18 +377,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
                 for (int c = 0; c < kBlockN / 32; ++c) {
-                    uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[c][i]), scale_log2, neg_m));
-                        const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 1]), scale_log2, neg_m));
-                        const float p2 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 2]), scale_log2, neg_m));
-                        const float p3 = ptx::ex2(fmaf(__uint_as_float(sv[c][i + 3]), scale_log2, neg_m));
-                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                        pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
-                        pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i]), scale_log2, neg_m));
+                            const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 1]), scale_log2, neg_m));
+                            const float p2 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 2]), scale_log2, neg_m));
+                            const float p3 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 3]), scale_log2, neg_m));
+                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                            pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
+                            pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
+                        }
+                        ptx::tmem_st8(t_s + c * 16 + h * 8, pk);
                     }
-                    ptx::tmem_st16(t_s + c * 16, pk);
                 }
                 l += (l0 + l1) + (l2 + l3);
                 ptx::tmem_wait_st();
@@ -401,6 +424,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
         }
+    }
+
+    else {
+        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();  // the idle warps of the last warpgroup
     }
 
     ptx::tc_fence_before();

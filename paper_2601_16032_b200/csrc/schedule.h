@@ -65,6 +65,9 @@ SAW_HD WorkItem decode_work(const SchedParams& p, long long k, int it) {
     w.backward = (p.sawtooth && (it & 1)) ? 1 : 0;
     const int n_kv = ceil_div_i(p.N, p.block_n);
     w.hi = 0;
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+#endif
     for (int q = 0; q < 2; ++q) {
         int h = 0;
         const int r = w.row0 + q * kBlockM;

@@ -1,0 +1,115 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what the header declares, validates
+arguments, and its host-side schedule replay agrees entry by entry with the schedule oracle."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2601_16032_b200 as sa
+from oracle import schedule as sch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    from paper_2601_16032_b200 import build
+    build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "sawtooth_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(attn_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(sa.library_path())
+    names = declared_functions()
+    assert {"attn_fwd", "attn_fwd_ex", "attn_fwd_host", "attn_query_plan", "attn_schedule_trace",
+            "attn_device_status", "attn_status_string", "attn_last_error"} <= set(names)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_status_strings():
+    assert sa.attn_status_string(0) == "ok"
+    for s in range(-6, 0):
+        assert sa.attn_status_string(s) not in ("ok", "unknown status")
+    assert sa.attn_status_string(-99) == "unknown status"
+
+
+def test_plan_matches_algorithm_2():
+    p = sa.attn_query_plan(4, 16, 8192, 128, 0, sa.BF16, sm_count=148)
+    assert (p.block_m, p.block_n, p.q_tiles, p.rows_per_item) == (128, 128, 2, 256)
+    assert p.items_per_head == 32 and p.n_work == 2048 and p.grid == 148  # G = min(N_tiles, N_SM)
+    assert p.smem_bytes <= 232448 and p.kv_stages >= 2
+    p = sa.attn_query_plan(1, 1, 1024, 64, 0, sa.F16, sm_count=148)
+    assert p.n_work == 4 and p.grid == 4
+    o = sa.Opts()
+    o.q_tiles, o.block_n, o.max_ctas = 1, 64, 5
+    p = sa.attn_query_plan(1, 8, 4096, 64, 0, sa.F16, o, sm_count=148)
+    assert (p.rows_per_item, p.block_n, p.n_work, p.grid) == (128, 64, 256, 5)
+    o = sa.Opts()
+    o.launch_mode = 1  # Algorithm 3: one CTA per work item
+    assert sa.attn_query_plan(1, 8, 4096, 64, 0, sa.F16, o, sm_count=148).grid == 128
+
+
+def test_argument_validation_without_a_device():
+    cases = [
+        (dict(B=0), -1), (dict(N=-3), -1), (dict(d=80), -2), (dict(causal=3), -1), (dict(dtype=9), -1),
+    ]
+    for change, status in cases:
+        a = dict(B=1, H=1, N=128, d=64, causal=0, dtype=0)
+        a.update(change)
+        with pytest.raises(sa.AttnError) as e:
+            sa.attn_query_plan(a["B"], a["H"], a["N"], a["d"], a["causal"], a["dtype"], sm_count=148)
+        assert e.value.status == status
+    bad = sa.Opts()
+    bad.block_n = 96
+    with pytest.raises(sa.AttnError):
+        sa.attn_query_plan(1, 1, 128, 64, 0, 0, bad, sm_count=148)
+    bad = sa.Opts()
+    bad.kv_stages = 99
+    with pytest.raises(sa.AttnError):
+        sa.attn_query_plan(1, 1, 128, 128, 0, 0, bad, sm_count=148)
+    with pytest.raises(sa.AttnError) as e:
+        sa.attn_fwd(0, 0, 0, 0, 1, 1, 128, 64, 0.125, 0, 0, 0)
+    assert e.value.status == -1 and "non-null" in str(e.value)
+
+
+SHAPES = [
+    # n_sm, B, H, N, d, q_tiles, block_n
+    (4, 1, 1, 1024, 64, 2, 128),
+    (148, 1, 8, 4096, 64, 2, 64),
+    (5, 2, 3, 1000, 128, 1, 64),
+    (7, 1, 2, 777, 128, 2, 128),
+    (148, 1, 1, 130, 64, 2, 128),
+    (3, 2, 2, 2049, 128, 2, 64),
+]
+
+
+@pytest.mark.parametrize("n_sm,B,H,N,d,q_tiles,block_n", SHAPES)
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("order", [sa.CYCLIC, sa.SAWTOOTH])
+@pytest.mark.parametrize("digits", [sa.TILE_FASTEST, sa.HEAD_FASTEST])
+def test_schedule_replay_equals_the_schedule_oracle(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits):
+    o = sa.Opts()
+    o.q_tiles, o.block_n, o.digit_order = q_tiles, block_n, digits
+    got = sa.attn_schedule_trace(B, H, N, d, causal, order, sa.F16, o, sm_count=n_sm)
+    W = 128 * q_tiles
+    want = [w for seq in sch.full_schedule(n_sm, B, H, N, W, block_n, bool(causal), order,
+                                           "head_fastest" if digits else "tile_fastest") for w in seq]
+    assert len(got) == len(want)
+    for g, w in zip(got, want):
+        assert (g.cta, g.iteration, g.k, g.batch, g.head, g.q_item, bool(g.backward), g.n_kv) == \
+            (w.cta, w.i_local, w.k, w.batch, w.head, w.q_tile, w.backward, w.n_kv)
+        # per 128-row tile ranges: what an item of W = 128 rows at that position would need
+        for qi, n_q in enumerate((g.n_kv_q0, g.n_kv_q1)):
+            r = g.q_item * W + qi * 128
+            if qi >= q_tiles or r >= N:
+                assert n_q == 0
+            else:
+                assert n_q == sch.kv_tiles_needed(r // 128, N, 128, block_n, bool(causal))
+        assert max(g.n_kv_q0, g.n_kv_q1) == g.n_kv
