@@ -137,9 +137,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const long long k_first = blockIdx.x;
     const long long k_stride = gridDim.x;
 
+    if (warp >= 4 * kQTiles) {
+    // The last warpgroup (producer, MMA and two idle warps) hands registers back in one instruction.
+    if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
         if (lane == 0) {
             uint64_t pol_kv = 0, pol_q = 0;
             if (p.l2_policy) { pol_kv = ptx::policy_evict_last(); pol_q = ptx::policy_evict_first(); }
@@ -196,7 +198,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue
-        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
         if (lane == 0) {
             constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
             constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
@@ -295,7 +296,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             drain_wait(&bar->drain, 0);
         }
         __syncwarp();
-    } else if (warp < 4 * kQTiles) {
+    }
+    } else {
         // ------------------------------------------------------------------ softmax / correction / epilogue
         if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
         const int q = warp >> 2;                       // which Q tile this warpgroup owns
@@ -426,9 +428,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     }
 
-    else {
-        if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();  // the idle warps of the last warpgroup
-    }
 
     ptx::tc_fence_before();
     __syncthreads();
