@@ -167,14 +167,19 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c3", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="c3", choices=sorted(wl.CONFIGS) + sorted(wl.STUDY_CASES))
+    ap.add_argument("--scan-order", default="both", choices=["both", "cyclic", "sawtooth"],
+                    help="orders to time; `value` is the sawtooth order unless only cyclic is timed")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--also", default="c2,c4,c5",
+                    help="further workloads timed briefly in both orders (single GPU only; '' for none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (default: min(steps, 10))")
     ap.add_argument("--cpu-heads", type=int, default=-1, help="heads the CPU baseline computes (default: sized to ~15 s)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    w = wl.CONFIGS[args.workload]
+    w = wl.CONFIGS.get(args.workload) or wl.STUDY_CASES[args.workload]
 
     if args.impl == "reference":
         run_reference(args, w)
@@ -195,7 +200,6 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     dev = torch.device("cuda", local)
-    tdt = torch.bfloat16 if w.dtype == wl.BF16 else torch.float16
     adt = sa.BF16 if w.dtype == wl.BF16 else sa.F16
     shape = (w.B, w.H, w.N, w.d)
     numel = w.B * w.H * w.N * w.d
@@ -215,9 +219,13 @@ def main():
     stream = torch.cuda.Stream(device=dev)
     sh = stream.cuda_stream
 
-    def step(order):
-        sa.attn_fwd(devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
-                    w.B, w.H, w.N, w.d, w.scale, int(w.causal), order, adt, sh)
+    def make_step(bufs, wk, a_dt):
+        def step(order):
+            sa.attn_fwd(bufs["q"].data_ptr(), bufs["k"].data_ptr(), bufs["v"].data_ptr(), bufs["o"].data_ptr(),
+                        wk.B, wk.H, wk.N, wk.d, wk.scale, int(wk.causal), order, a_dt, sh)
+        return step
+
+    step = make_step(devb, w, adt)
 
     def barrier():
         if dist is not None:
@@ -225,6 +233,7 @@ def main():
         torch.cuda.synchronize(dev)
 
     def timed(fn, steps):
+        """Milliseconds of `steps` calls of fn on the launch stream (CUDA events), max over ranks."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         with torch.cuda.stream(stream):
@@ -240,28 +249,72 @@ def main():
             ms = float(t.item())
         return ms
 
+    orders = {"cyclic": sa.CYCLIC, "sawtooth": sa.SAWTOOTH}
+    timed_orders = ["cyclic", "sawtooth"] if args.scan_order == "both" else [args.scan_order]
+    headline = "sawtooth" if "sawtooth" in timed_orders else "cyclic"
     results = {}
     with ClockSampler(local) as clocks:
-        for order, name in ((sa.CYCLIC, "cyclic"), (sa.SAWTOOTH, "sawtooth")):
+        for name in timed_orders:
             for _ in range(args.warmup):
-                step(order)
-            ms = timed(lambda: step(order), args.steps)
-            results[name] = ms / args.steps
+                step(orders[name])
+            results[name] = timed(lambda: step(orders[name]), args.steps) / args.steps
     sa.attn_device_status()
     clk = clocks.summary()
 
+    # The two orders launch by launch in alternation, so that neither sees a hotter or a cooler GPU.
+    ab = None
+    if len(timed_orders) == 2:
+        pairs = max(3, min(args.steps, 20))
+        acc = {"cyclic": [], "sawtooth": []}
+        for _ in range(pairs):
+            for name in timed_orders:
+                acc[name].append(timed(lambda: step(orders[name]), 1))
+        ab = {n: float(np.median(v)) for n, v in acc.items()}
+
     # End to end: host buffers in, host buffer out, copies inside the timed region.
-    e2e_steps = args.e2e_steps or min(args.steps, 10)
+    e2e = None
+    if not args.skip_e2e:
+        e2e_steps = args.e2e_steps or min(args.steps, 10)
 
-    def e2e_step():
-        sa.attn_fwd_host(host["q"].data_ptr(), host["k"].data_ptr(), host["v"].data_ptr(), host["o"].data_ptr(),
-                         devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
-                         w.B, w.H, w.N, w.d, w.scale, int(w.causal), sa.SAWTOOTH, adt, sh)
+        def e2e_step():
+            sa.attn_fwd_host(host["q"].data_ptr(), host["k"].data_ptr(), host["v"].data_ptr(), host["o"].data_ptr(),
+                             devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
+                             w.B, w.H, w.N, w.d, w.scale, int(w.causal), orders[headline], adt, sh)
 
-    for _ in range(2):
-        e2e_step()
-    e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
-    sa.attn_device_status()
+        for _ in range(2):
+            e2e_step()
+        e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
+        sa.attn_device_status()
+        e2e = {"value": w.flops / e2e_ms / 1e9 * world, "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "h2d_bytes_per_step": 3 * numel * 2, "d2h_bytes_per_step": numel * 2}
+
+    # The other configurations, timing only (inputs drawn on the device from a seed), single GPU only.
+    also = {}
+    if world == 1 and args.also:
+        del devb
+        torch.cuda.empty_cache()
+        for name in [n for n in args.also.split(",") if n]:
+            wk = wl.CONFIGS.get(name) or wl.STUDY_CASES[name]
+            tdt = torch.bfloat16 if wk.dtype == wl.BF16 else torch.float16
+            g = torch.Generator(device=dev).manual_seed(wk.seed)
+            bufs = {}
+            for n in ("q", "k", "v"):
+                bufs[n] = torch.randn((wk.B, wk.H, wk.N, wk.d), device=dev, generator=g, dtype=torch.float32).to(tdt)
+            if wk.k_scale != 1.0:
+                bufs["k"] *= wk.k_scale
+            bufs["o"] = torch.empty_like(bufs["q"])
+            st = make_step(bufs, wk, sa.BF16 if wk.dtype == wl.BF16 else sa.F16)
+            n_steps = max(3, min(args.steps, int(200.0 / (wk.flops / 1e12))))  # about 0.2 s per order
+            entry = {"workload": config_of(wk)["workload"], "steps": n_steps}
+            for oname in ("cyclic", "sawtooth"):
+                for _ in range(3):
+                    st(orders[oname])
+                ms = timed(lambda: st(orders[oname]), n_steps) / n_steps
+                entry[oname] = {"value": wk.flops / ms / 1e9, "unit": UNIT, "ms_per_step": ms}
+            sa.attn_device_status()
+            also[name] = entry
+            del bufs
+            torch.cuda.empty_cache()
 
     if rank != 0:
         if dist is not None:
@@ -270,33 +323,38 @@ def main():
 
     peaks = measured_peaks()
     flops = w.flops
-    ms_saw, ms_cyc = results["sawtooth"], results["cyclic"]
-    tf_saw = flops / ms_saw / 1e9
-    tf_cyc = flops / ms_cyc / 1e9
-    timed_region_s = ms_saw * args.steps / 1e3
+    ms_head = results[headline]
+    tf_head = flops / ms_head / 1e9
+    timed_region_s = ms_head * args.steps / 1e3
     peak_kind = "sustained" if timed_region_s >= 0.5 else "burst"
     peak = peaks[peak_kind]
     plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt)
     line = {
-        "metric": METRIC, "value": tf_saw * world, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_saw, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": tf_head * world, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_head, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == wl.BF16 else "f16", "data": "synthetic",
-        "config": config_of(w, {"scan_order": "sawtooth", "parallelism": "replicas only" if world > 1 else "single GPU",
+        "config": config_of(w, {"scan_order": headline, "parallelism": "replicas only" if world > 1 else "single GPU",
                                 "grid": plan.grid, "rows_per_item": plan.rows_per_item, "block_n": plan.block_n,
                                 "kv_stages": plan.kv_stages}),
-        "cyclic": {"value": tf_cyc * world, "unit": UNIT, "ms_per_step": ms_cyc},
-        "sawtooth_over_cyclic": tf_saw / tf_cyc,
         "clocks": clk,
-        "e2e": {"value": flops / e2e_ms / 1e9 * world, "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                "h2d_bytes_per_step": 3 * numel * 2, "d2h_bytes_per_step": numel * 2},
         "gpu_launches": args.steps,
-        "roofline": {"bound": "tensor", "achieved": tf_saw, "peak": peak, "unit": UNIT, "frac": tf_saw / peak,
+        "roofline": {"bound": "tensor", "achieved": tf_head, "peak": peak, "unit": UNIT, "frac": tf_head / peak,
                      "peak_kind": f"{peak_kind} bf16 matmul, of {peaks['source']}",
-                     "frac_of_burst": tf_saw / peaks["burst"], "frac_of_sustained": tf_saw / peaks["sustained"],
-                     "frac_of_nominal_2250": tf_saw / NOMINAL_BF16_TFLOPS,
-                     "flops_per_launch": flops, "launch_ms": ms_saw,
+                     "frac_of_burst": tf_head / peaks["burst"], "frac_of_sustained": tf_head / peaks["sustained"],
+                     "frac_of_nominal_2250": tf_head / NOMINAL_BF16_TFLOPS,
+                     "flops_per_launch": flops, "launch_ms": ms_head,
                      "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name), "compulsory_bytes": w.compulsory_bytes},
     }
+    if e2e is not None:
+        line["e2e"] = e2e
+    for name in timed_orders:
+        if name != headline:
+            line[name] = {"value": flops / results[name] / 1e9 * world, "unit": UNIT, "ms_per_step": results[name]}
+    if ab is not None:
+        line["alternating_launches"] = {"cyclic_ms": ab["cyclic"], "sawtooth_ms": ab["sawtooth"],
+                                        "sawtooth_over_cyclic": ab["cyclic"] / ab["sawtooth"]}
+    if also:
+        line["also"] = also
     if not args.skip_cpu_baseline:
         from oracle import attention as ora
         per_head_flops = 4.0 * float(w.N) ** 2 * w.d / (2 if w.causal else 1)

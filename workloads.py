@@ -60,6 +60,16 @@ CONFIGS = {
     "c5": Workload("c5", 2, 16, 65536, 128, BF16, True, 1005),
 }
 
+# Smaller or differently shaped cases for profiler captures and scan-order studies (not parity
+# configurations).  "long*" follow the paper's own studies: a single head whose K+V exceeds L2.
+STUDY_CASES = {
+    "c3-small": Workload("c3-small", 2, 16, 8192, 128, BF16, False, 2003),
+    "c4-small": Workload("c4-small", 1, 8, 32768, 128, BF16, True, 2004, k_scale=0.5),
+    "long-256k": Workload("long-256k", 1, 1, 262144, 128, BF16, False, 2006),
+    "long-512k": Workload("long-512k", 1, 1, 524288, 128, BF16, False, 2007),
+    "long-128k-b8": Workload("long-128k-b8", 8, 1, 131072, 64, F16, False, 2008),
+}
+
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round fp32 to bfloat16 (nearest, ties to even) and return the 16-bit patterns."""
