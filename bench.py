@@ -106,6 +106,22 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(ms: float, dist=None, device=None) -> float:
+    """The slowest rank's time: what the whole job took.  `dist` is torch.distributed once a process
+    group exists (any backend), else None for a single process."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank: float, ms: float, world: int) -> float:
+    """Independent replicas: every rank does the same work, the job lasts as long as its slowest rank."""
+    return flops_per_rank * world / ms / 1e9
+
+
 def oracle_sample_heads(w: wl.Workload, n_heads: int):
     return list(wl.all_heads(w))[:n_heads]
 
@@ -242,12 +258,7 @@ def main():
                 fn()
             e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     orders = {"cyclic": sa.CYCLIC, "sawtooth": sa.SAWTOOTH}
     timed_orders = ["cyclic", "sawtooth"] if args.scan_order == "both" else [args.scan_order]
@@ -285,7 +296,7 @@ def main():
             e2e_step()
         e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
         sa.attn_device_status()
-        e2e = {"value": w.flops / e2e_ms / 1e9 * world, "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+        e2e = {"value": whole_job_tflops(w.flops, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
                "h2d_bytes_per_step": 3 * numel * 2, "d2h_bytes_per_step": numel * 2}
 
     # The other configurations, timing only (inputs drawn on the device from a seed), single GPU only.
@@ -324,13 +335,13 @@ def main():
     peaks = measured_peaks()
     flops = w.flops
     ms_head = results[headline]
-    tf_head = flops / ms_head / 1e9
+    tf_head = whole_job_tflops(flops, ms_head, 1)  # one GPU's throughput; `value` is the job's
     timed_region_s = ms_head * args.steps / 1e3
     peak_kind = "sustained" if timed_region_s >= 0.5 else "burst"
     peak = peaks[peak_kind]
     plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt)
     line = {
-        "metric": METRIC, "value": tf_head * world, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC, "value": whole_job_tflops(flops, ms_head, world), "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_head, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == wl.BF16 else "f16", "data": "synthetic",
         "config": config_of(w, {"scan_order": headline, "parallelism": "replicas only" if world > 1 else "single GPU",
@@ -349,7 +360,7 @@ def main():
         line["e2e"] = e2e
     for name in timed_orders:
         if name != headline:
-            line[name] = {"value": flops / results[name] / 1e9 * world, "unit": UNIT, "ms_per_step": results[name]}
+            line[name] = {"value": whole_job_tflops(flops, results[name], world), "unit": UNIT, "ms_per_step": results[name]}
     if ab is not None:
         line["alternating_launches"] = {"cyclic_ms": ab["cyclic"], "sawtooth_ms": ab["sawtooth"],
                                         "sawtooth_over_cyclic": ab["cyclic"] / ab["sawtooth"]}

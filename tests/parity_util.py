@@ -44,25 +44,40 @@ def output_bits(o, b: int, h: int, rows=None) -> np.ndarray:
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def compare_with_oracle(w: wl.Workload, o, plan=None):
-    """Returns (max_abs, mean_abs, n_rows) of the CUDA output against the oracle on the planned rows."""
+def _head_f64(w: wl.Workload, b: int, h: int):
+    return tuple(wl.bits_to_f64(wl.head_bits(w, n, b, h), w.dtype) for n in ("q", "k", "v"))
+
+
+def oracle_rows(w: wl.Workload, plan) -> dict:
+    """The oracle's output for the planned rows: {(b, h): (row indices, [n_rows, d] fp64)}."""
     from oracle import attention as ora
-    plan = plan if plan is not None else wl.checked_rows(w)
+    want = {}
+    for (b, h), rows in plan.items():
+        q, k, v = _head_f64(w, b, h)
+        idx = np.arange(w.N, dtype=np.int64) if rows is None else np.asarray(rows, dtype=np.int64)
+        want[(b, h)] = (idx, ora.attention_rows(q[idx], idx, k, v, w.scale, w.causal))
+    return want
+
+
+def compare_rows(w: wl.Workload, o, plan, want):
+    """(max_abs, mean_abs, n_rows) of the CUDA output `o` against precomputed oracle rows."""
     max_abs, total, count, n_rows = 0.0, 0.0, 0, 0
     for (b, h), rows in plan.items():
-        q = wl.bits_to_f64(wl.head_bits(w, "q", b, h), w.dtype)
-        k = wl.bits_to_f64(wl.head_bits(w, "k", b, h), w.dtype)
-        v = wl.bits_to_f64(wl.head_bits(w, "v", b, h), w.dtype)
-        idx = np.arange(w.N, dtype=np.int64) if rows is None else np.asarray(rows, dtype=np.int64)
-        want = ora.attention_rows(q[idx], idx, k, v, w.scale, w.causal)
+        idx, ref = want[(b, h)]
         got = wl.bits_to_f64(output_bits(o, b, h, None if rows is None else idx), w.dtype)
         assert np.isfinite(got).all(), f"non-finite output in head ({b},{h})"
-        err = np.abs(got - want)
+        err = np.abs(got - ref)
         max_abs = max(max_abs, float(err.max()))
         total += float(err.sum())
         count += err.size
         n_rows += len(idx)
     return max_abs, total / count, n_rows
+
+
+def compare_with_oracle(w: wl.Workload, o, plan=None):
+    """Returns (max_abs, mean_abs, n_rows) of the CUDA output against the oracle on the planned rows."""
+    plan = plan if plan is not None else wl.checked_rows(w)
+    return compare_rows(w, o, plan, oracle_rows(w, plan))
 
 
 def assert_parity(w: wl.Workload, o, plan=None):

@@ -1,0 +1,62 @@
+"""GPU parity on the five benchmark configurations at full size, through the C ABI, in the launch
+configuration the benchmark times (library defaults), both scan orders.
+
+The oracle result of the checked rows is computed once per configuration and both orders are
+compared with it: every row of every head for c1 and c2, every row of two heads plus seeded rows
+elsewhere for c3 and c4, 512 seeded rows plus the tile-edge rows in every head for c5."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from parity_util import MAX_ABS_TOL, MEAN_ABS_TOL, oracle_rows, compare_rows, run_cuda, upload, output_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def check_config(name, opts_list):
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.CONFIGS[name]
+    plan = wl.checked_rows(w)
+    want = oracle_rows(w, plan)
+    qkv = upload(w)
+    outs = {}
+    for label, opts in opts_list:
+        for order in (sa.CYCLIC, sa.SAWTOOTH):
+            o = run_cuda(w, qkv, order, opts)
+            max_abs, mean_abs, n_rows = compare_rows(w, o, plan, want)
+            assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, \
+                f"{name} {label} order {order}: max_abs {max_abs:.3e} mean_abs {mean_abs:.3e} over {n_rows} rows"
+            outs[(label, order)] = o if w.compulsory_bytes <= (64 << 20) else None
+            del o
+    torch.cuda.empty_cache()
+    return w, outs
+
+
+def test_c1_all_rows_both_tile_shapes():
+    import paper_2601_16032_b200 as sa
+    o64 = sa.Opts()
+    o64.block_n = 64
+    w, outs = check_config("c1", [("default", None), ("128x64", o64)])
+    a = wl.bits_to_f64(output_bits(outs[("default", sa.CYCLIC)], 0, 0), w.dtype)
+    b = wl.bits_to_f64(output_bits(outs[("default", sa.SAWTOOTH)], 0, 0), w.dtype)
+    assert np.abs(a - b).max() <= 1e-2
+
+
+def test_c2_all_rows_128x64_tiles_and_default():
+    import paper_2601_16032_b200 as sa
+    o64 = sa.Opts()
+    o64.block_n = 64  # the 128 x 64 Q / K tiles this configuration names
+    check_config("c2", [("128x64", o64), ("default", None)])
+
+
+def test_c3_two_heads_plus_sampled_rows():
+    check_config("c3", [("default", None)])
+
+
+def test_c4_causal_two_heads_plus_sampled_rows():
+    check_config("c4", [("default", None)])
+
+
+def test_c5_causal_sampled_rows_every_head():
+    check_config("c5", [("default", None)])
