@@ -28,6 +28,10 @@ struct KernelParams {
 };
 
 constexpr int kMaxStages = 16;
+#ifndef SAW_EXP_POLY_OF_4
+#define SAW_EXP_POLY_OF_4 0
+#endif
+constexpr int kExpPolyOf4 = SAW_EXP_POLY_OF_4;  // of every four pairs of exponentials, how many avoid the MUFU
 constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the row max grew by more (log2 units)
 
 // Codes written to the status word: which wait gave up.
@@ -142,17 +146,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint64_t pol_kv = 0, pol_q = 0;
-            if (p.l2_policy) { pol_kv = ptx::policy_evict_last(); pol_q = ptx::policy_evict_first(); }
-            Ring ring;
-            uint32_t q_issued = 0;     // Q loads issued so far
-            long long kv_issued = 0;   // K/V tile loads issued so far
-            bool ok = true;
-            int it = 0;
-            for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
-                const WorkItem w = decode_work(p.sched, k, it);
-                if (!ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ)) { ok = false; break; }
+        // The whole warp walks the schedule and waits on the barriers; one elected lane issues the
+        // copies (elect.sync keeps the issue path warp-uniform for the compiler).
+        uint64_t pol_kv = 0, pol_q = 0;
+        if (p.l2_policy) { pol_kv = ptx::policy_evict_last(); pol_q = ptx::policy_evict_first(); }
+        Ring ring;
+        uint32_t q_issued = 0;     // Q loads issued so far
+        long long kv_issued = 0;   // K/V tile loads issued so far
+        bool ok = true;
+        int it = 0;
+        for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+            const WorkItem w = decode_work(p.sched, k, it);
+            ok = ptx::warp_all(ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ));
+            if (!ok) break;
+            if (ptx::elect_one()) {
                 int n_valid = 0;
 #pragma unroll
                 for (int q = 0; q < kQTiles; ++q) n_valid += (w.hi_q[q] > 0);
@@ -167,78 +174,86 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         else ptx::tma_load_3d(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh);
                     }
                 }
-                ++q_issued;
-                for (int s = 0; ok && s < w.hi; ++s) {
-                    const int j = kv_tile_at(w, s);
-                    for (int kv = 0; kv < 2; ++kv) {
-                        if (!ptx::mbar_wait(&bar->kv_empty[ring.slot], ring.phase ^ 1u, abort_flag, kSiteProducerKV)) { ok = false; break; }
+            }
+            __syncwarp();
+            ++q_issued;
+            for (int s = 0; ok && s < w.hi; ++s) {
+                const int j = kv_tile_at(w, s);
+                for (int kv = 0; kv < 2; ++kv) {
+                    ok = ptx::warp_all(ptx::mbar_wait(&bar->kv_empty[ring.slot], ring.phase ^ 1u, abort_flag, kSiteProducerKV));
+                    if (!ok) break;
+                    if (ptx::elect_one()) {
                         ptx::mbar_arrive_expect_tx(&bar->kv_full[ring.slot], G::kKVTileBytes);
                         const CUtensorMap* tm = kv ? &tm_v : &tm_k;
+#pragma unroll
                         for (int c = 0; c < G::kChunks; ++c) {
                             void* dst = kv_smem + (size_t)ring.slot * G::kKVTileBytes + c * G::kKVChunkBytes;
                             if (p.l2_policy) ptx::tma_load_3d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh, pol_kv);
                             else ptx::tma_load_3d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh);
                         }
-                        ring.advance(stages);
-                        ++kv_issued;
                     }
+                    __syncwarp();
+                    ring.advance(stages);
+                    ++kv_issued;
                 }
             }
-            if (!ok) {
-                // Leave no copy in flight: wait (briefly) for the loads issued last into each slot.
-                if (q_issued) drain_wait(&bar->q_full, (q_issued - 1) & 1u);
-                const int back = kv_issued < stages ? (int)kv_issued : stages;
-                Ring r = ring;
-                for (int n = 0; n < back; ++n) {
-                    if (r.slot == 0) { r.slot = stages - 1; r.phase ^= 1u; } else { --r.slot; }
-                    drain_wait(&bar->kv_full[r.slot], r.phase);
-                }
+        }
+        if (!ok) {
+            // Leave no copy in flight: wait (briefly) for the loads issued last into each slot.
+            if (q_issued) drain_wait(&bar->q_full, (q_issued - 1) & 1u);
+            const int back = kv_issued < stages ? (int)kv_issued : stages;
+            Ring r = ring;
+            for (int n = 0; n < back; ++n) {
+                if (r.slot == 0) { r.slot = stages - 1; r.phase ^= 1u; } else { --r.slot; }
+                drain_wait(&bar->kv_full[r.slot], r.phase);
             }
         }
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issue
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
-            constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
-            const uint32_t q_base = ptx::smem_u32(q_smem);
-            const uint32_t kv_base = ptx::smem_u32(kv_smem);
-            Ring ring;
-            uint32_t p_phase[2] = {0, 0};
-            bool ok = true;
+        constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
+        constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
+        const uint32_t q_base = ptx::smem_u32(q_smem);
+        const uint32_t kv_base = ptx::smem_u32(kv_smem);
+        Ring ring;
+        uint32_t p_phase[2] = {0, 0};
+        bool ok = true;
 
-            // Descriptors differ from a base only in the 16-byte-granular address field (the low bits).
-            const uint64_t q_desc0 = ptx::smem_desc_sw128(q_base, 16, 1024);
-            const uint64_t k_desc0 = ptx::smem_desc_sw128(kv_base, 16, 1024);
-            const uint64_t v_desc0 = ptx::smem_desc_sw128(kv_base, G::kKVChunkBytes, 1024);
-            auto issue_qk = [&](int q, int slot) {
-                const uint64_t a0 = q_desc0 + (uint64_t)((q * G::kQTileBytes) >> 4);
-                const uint64_t b0 = k_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
-                const uint32_t d_tmem = tmem + G::kTmemS + 128 * q;
+        // Descriptors differ from a base only in the 16-byte-granular address field (the low bits).
+        const uint64_t q_desc0 = ptx::smem_desc_sw128(q_base, 16, 1024);
+        const uint64_t k_desc0 = ptx::smem_desc_sw128(kv_base, 16, 1024);
+        const uint64_t v_desc0 = ptx::smem_desc_sw128(kv_base, G::kKVChunkBytes, 1024);
+        auto issue_qk = [&](int q, int slot) {
+            const uint64_t a0 = q_desc0 + (uint64_t)((q * G::kQTileBytes) >> 4);
+            const uint64_t b0 = k_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
+            const uint32_t d_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
-                for (int i = 0; i < G::kChunks * 4; ++i) {
-                    const int c = i >> 2, kk = i & 3;
-                    ptx::mma_ss(d_tmem, a0 + (uint64_t)((c * G::kQChunkBytes + kk * 32) >> 4),
-                                b0 + (uint64_t)((c * G::kKVChunkBytes + kk * 32) >> 4), idesc_qk, i != 0);
-                }
-            };
-            auto issue_pv = [&](int q, int slot, uint32_t accumulate) {
-                const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
-                const uint32_t d_tmem = tmem + G::kTmemO + 128 * q;
-                const uint32_t a_tmem = tmem + G::kTmemS + 128 * q;
+            for (int i = 0; i < G::kChunks * 4; ++i) {
+                const int c = i >> 2, kk = i & 3;
+                ptx::mma_ss(d_tmem, a0 + (uint64_t)((c * G::kQChunkBytes + kk * 32) >> 4),
+                            b0 + (uint64_t)((c * G::kKVChunkBytes + kk * 32) >> 4), idesc_qk, i != 0);
+            }
+        };
+        auto issue_pv = [&](int q, int slot, uint32_t accumulate) {
+            const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
+            const uint32_t d_tmem = tmem + G::kTmemO + 128 * q;
+            const uint32_t a_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
-                for (int kk = 0; kk < kBlockN / 16; ++kk) {
-                    ptx::mma_ts(d_tmem, a_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
-                                accumulate | (kk != 0));
-                }
-            };
+            for (int kk = 0; kk < kBlockN / 16; ++kk) {
+                ptx::mma_ts(d_tmem, a_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
+                            accumulate | (kk != 0));
+            }
+        };
 
+        // One elected lane runs the whole loop: every wait, issue and commit below is a single
+        // thread's, with no warp votes or re-convergence between the MMA batches.
+        if (ptx::elect_one()) {
             int it = 0;
             for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
                 const WorkItem w = decode_work(p.sched, k, it);
                 if (!ptx::mbar_wait(&bar->q_full, it & 1, abort_flag, kSiteMmaQ)) { ok = false; break; }
                 // K tile of step 0
-                int slot_k = ring.slot;
+                const int slot_k = ring.slot;
                 if (!ptx::mbar_wait(&bar->kv_full[slot_k], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                 ring.advance(stages);
                 ptx::tc_fence_after();
@@ -376,7 +391,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                const ptx::f32x2 scale2 = ptx::pack_f32x2(scale_log2, scale_log2);
+                const ptx::f32x2 neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
+                ptx::f32x2 l01 = ptx::pack_f32x2(0.f, 0.f), l23 = ptx::pack_f32x2(0.f, 0.f);
 #pragma unroll
                 for (int c = 0; c < kBlockN / 32; ++c) {
 #pragma unroll
@@ -384,17 +401,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         uint32_t pk[8];
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {
-                            const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i]), scale_log2, neg_m));
-                            const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 1]), scale_log2, neg_m));
-                            const float p2 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 2]), scale_log2, neg_m));
-                            const float p3 = ptx::ex2(fmaf(__uint_as_float(sv[c][16 * h + i + 3]), scale_log2, neg_m));
-                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                            // Four probabilities: x = S * scale * log2(e) - m as two packed FMAs, then 2^x on the MUFU
+                            // or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
+                            const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
+                            const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
+                            float x0, x1, x2, x3, p0, p1, p2, p3;
+                            ptx::unpack_f32x2(xa, x0, x1);
+                            ptx::unpack_f32x2(xb, x2, x3);
+                            if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
+                            else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
+                            if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
+                            else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
+                            l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
+                            l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
                             pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
                             pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
                         }
                         ptx::tmem_st8(t_s + c * 16 + h * 8, pk);
                     }
                 }
+                float l0, l1, l2, l3;
+                ptx::unpack_f32x2(l01, l0, l1);
+                ptx::unpack_f32x2(l23, l2, l3);
                 l += (l0 + l1) + (l2 + l3);
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();

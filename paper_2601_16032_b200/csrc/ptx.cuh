@@ -19,6 +19,20 @@ __device__ __forceinline__ uint32_t lane_id() {
     return l;
 }
 
+// True in exactly one lane of a fully converged warp (the same lane on every call).  Code guarded by
+// it is known to the compiler to run in a single lane, so instructions that take warp-uniform
+// operands (TMA, MMA issue) are generated without a per-lane loop.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ bool warp_all(bool x) { return __all_sync(0xffffffffu, x) != 0; }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -247,6 +261,59 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed pairs of fp32 (one 64-bit register): sm_100 executes one f32x2 instruction for two lanes' worth
+// of FMA-pipe work.
+typedef uint64_t f32x2;
+__device__ __forceinline__ f32x2 pack_f32x2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2_round_down(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// 2^x for a pair, x <= 127, on the FMA and ALU pipes instead of the MUFU.  x is clamped below at
+// -126, split into floor(x) (taken from the low mantissa bits of x + 1.5*2^23 rounded down) and
+// the fraction f in [0, 1); 2^f comes from a cubic with minimax relative error 7.5e-5 on [0, 1]
+// (Remez exchange on (p(f) - 2^f) / 2^f), well below the rounding of the 16-bit probabilities it
+// feeds; floor(x) is then added into the exponent field.
+__device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float& y0, float& y1) {
+    const float kMagic = 12582912.f;  // 1.5 * 2^23
+    const f32x2 magic = pack_f32x2(kMagic, kMagic);
+    const f32x2 x = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const f32x2 t = add2_round_down(x, magic);
+    const f32x2 f = sub2(x, sub2(t, magic));
+    f32x2 pl = fma2(f, pack_f32x2(0.07802452147006989f, 0.07802452147006989f), pack_f32x2(0.22606715559959412f, 0.22606715559959412f));
+    pl = fma2(pl, f, pack_f32x2(0.6958335638046265f, 0.6958335638046265f));
+    pl = fma2(pl, f, pack_f32x2(0.9999251961708069f, 0.9999251961708069f));
+    float t0, t1, p0, p1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(pl, p0, p1);
+    y0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+    y1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+}
+
 // Two fp32 -> one packed pair of 16-bit values (round to nearest even); `lo` lands in the low half.
 template <int kBf16>
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
