@@ -34,7 +34,7 @@ struct Resolved {
 };
 
 size_t smem_for(int d, int block_n, int q_tiles, int stages) {
-    return 1024 + (size_t)q_tiles * kBlockM * d * 2 + (size_t)stages * block_n * d * 2 + sizeof(Barriers);
+    return (size_t)q_tiles * kBlockM * d * 2 + (size_t)stages * block_n * d * 2 + sizeof(Barriers);
 }
 
 int check_shape(int B, int H, int N, int d, int causal, int dtype) {
@@ -204,7 +204,7 @@ int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const att
     out->items_per_head = sp.n_q;
     out->n_work = sp.n_work;
     out->grid = grid_for(sp.n_work, sm_count, r);
-    out->threads = r.q_tiles * 128 + 128;
+    out->threads = r.q_tiles * 128 * SAW_THREADS_PER_ROW + 128;
     out->kv_stages = r.stages;
     out->smem_bytes = (int)r.smem;
     out->sm_count = sm_count;

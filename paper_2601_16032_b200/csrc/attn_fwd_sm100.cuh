@@ -2,16 +2,20 @@
 // S, P and O in tensor memory, one softmax thread per query row.
 //
 // One CTA handles work items of kQTiles x 128 query rows (Algorithm 1's resident Q tile).  Warp roles:
-//   warps [0, 4*kQTiles)   softmax: warpgroup q owns the 128 rows of Q tile q, thread r owns row r
-//                          (TMEM lane r): reads S from TMEM, keeps the running max and sum, writes
-//                          P back to TMEM as 16-bit pairs, rescales O when the max moved, and at the
-//                          end of the item normalises O and stores it.
-//   warp 4*kQTiles         producer: one lane issues the TMA loads (Q tiles, then K_j, V_j in the
-//                          scan order of the item) into a ring of shared-memory slots.
-//   warp 4*kQTiles + 1     MMA: one lane issues S_q = Q_q K_j^T and O_q += P_q V_j and commits them
-//                          to mbarriers; the warp also owns the TMEM allocation.
+//   warps [0, 8*kQTiles)   softmax: two warpgroups per Q tile; row r of the tile (TMEM lane r) is shared
+//                          by two threads, one per half of the K/V tile's columns.  Each reads its half
+//                          of S from TMEM, the two exchange their row maxima through shared memory,
+//                          keep the running max and a partial sum, write P back to TMEM as 16-bit
+//                          pairs, rescale their half of O's columns when the max moved, and at the end
+//                          of the item normalise and store their half of the O row.
+//   warp 8*kQTiles         producer: one elected lane issues the TMA loads (Q tiles, then K_j, V_j in
+//                          the scan order of the item) into a ring of shared-memory slots.
+//   warp 8*kQTiles + 1     MMA: one elected lane issues S_q = Q_q K_j^T and O_q += P_q V_j and commits
+//                          them to mbarriers; the warp also owns the TMEM allocation.
 //   two more warps         idle; they complete the warpgroup whose registers go to the softmax threads.
 // With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
+// Four softmax warps per scheduler (two threads per row) keep the MUFU busy: one warp alone can start
+// an exponential only every other MUFU slot.
 #pragma once
 #include "ptx.cuh"
 #include "schedule.h"
@@ -28,6 +32,9 @@ struct KernelParams {
 };
 
 constexpr int kMaxStages = 16;
+#ifndef SAW_THREADS_PER_ROW
+#define SAW_THREADS_PER_ROW 2
+#endif
 #ifndef SAW_EXP_POLY_OF_4
 #define SAW_EXP_POLY_OF_4 0
 #endif
@@ -37,7 +44,7 @@ constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the
 // Codes written to the status word: which wait gave up.
 enum WaitSite {
     kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
-    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7
+    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8
 };
 
 struct __align__(8) Barriers {
@@ -47,6 +54,7 @@ struct __align__(8) Barriers {
     uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
+    float xchg[2][2][128];  // [Q tile][column half][row]: row maxima, and the partial row sums at the end of an item
 };
 
 template <int kD, int kBlockN, int kQTiles>
@@ -56,19 +64,24 @@ struct Geometry {
     static constexpr int kKVTileBytes = kBlockN * kD * 2;
     static constexpr int kQChunkBytes = kBlockM * 128;
     static constexpr int kKVChunkBytes = kBlockN * 128;
-    static constexpr int kSoftmaxThreads = kQTiles * 128;
-    static constexpr int kThreads = kSoftmaxThreads + 128;  // a full fourth/third warpgroup: producer, MMA, two idle warps
-    // Registers: the launch gives every thread 65536 / kThreads (rounded down to a multiple of 8).  With
-    // two Q tiles that is 168, too few for a softmax thread holding a 128-wide score row, so the last
-    // warpgroup hands registers back and the softmax warpgroups take them.
+    static constexpr int kSplit = SAW_THREADS_PER_ROW;      // threads per query row (1 or 2)
+    static constexpr int kColsS = kBlockN / kSplit;         // S columns a softmax thread owns
+    static constexpr int kColsO = kD / kSplit;              // O columns a softmax thread owns
+    static constexpr int kSoftmaxWarps = kQTiles * kSplit * 4;
+    static constexpr int kTileThreads = 128 * kSplit;       // threads that share one Q tile (one named barrier)
+    static constexpr int kThreads = kSoftmaxWarps * 32 + 128;  // plus one warpgroup: producer, MMA, two idle warps
+    // Registers: the launch gives every thread 65536 / kThreads rounded down to a multiple of 8.  With
+    // two Q tiles that is 96 (640 threads, two per row) or 168 (384 threads, one per row): the last
+    // warpgroup hands registers back and the softmax warpgroups take them
+    // (512 * 104 + 128 * 64 = 640 * 96; 256 * 200 + 128 * 104 = 384 * 168).
     static constexpr bool kRebalance = (kQTiles == 2);
-    static constexpr int kRegsOther = 104;
-    static constexpr int kRegsSoftmax = 200;
+    static constexpr int kRegsOther = kSplit == 2 ? 64 : 104;
+    static constexpr int kRegsSoftmax = kSplit == 2 ? 104 : 200;
     static constexpr int kTmemCols = 512;
     static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q aliases its first kBlockN/2 columns
     static constexpr int kTmemO = 256;    // O_q (fp32, kD columns) at kTmemO + 128 q
     static constexpr size_t smem_bytes(int stages) {
-        return 1024 + (size_t)kQTiles * kQTileBytes + (size_t)stages * kKVTileBytes + sizeof(Barriers);
+        return (size_t)kQTiles * kQTileBytes + (size_t)stages * kKVTileBytes + sizeof(Barriers);
     }
 };
 
@@ -94,8 +107,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const __grid_constant__ CUtensorMap tm_v, const KernelParams p)
 {
     using G = Geometry<kD, kBlockN, kQTiles>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if ((ptx::smem_u32(smem) & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)kSiteSmemAlignment);
+        return;
+    }
     uint8_t* q_smem = smem;
     uint8_t* kv_smem = smem + kQTiles * G::kQTileBytes;
     Barriers* bar = reinterpret_cast<Barriers*>(kv_smem + (size_t)p.kv_stages * G::kKVTileBytes);
@@ -104,8 +120,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-    constexpr int kProducerWarp = 4 * kQTiles;
-    constexpr int kMmaWarp = 4 * kQTiles + 1;
+    constexpr int kProducerWarp = G::kSoftmaxWarps;
+    constexpr int kMmaWarp = G::kSoftmaxWarps + 1;
     const int stages = p.kv_stages;
 
     if (tid == 0) {
@@ -117,7 +133,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         for (int q = 0; q < 2; ++q) {
             ptx::mbar_init(&bar->s_full[q], 1);
-            ptx::mbar_init(&bar->p_full[q], 128);
+            ptx::mbar_init(&bar->p_full[q], G::kTileThreads);
             ptx::mbar_init(&bar->o_full[q], 1);
         }
         ptx::mbar_init(&bar->drain, 1);
@@ -141,7 +157,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const long long k_first = blockIdx.x;
     const long long k_stride = gridDim.x;
 
-    if (warp >= 4 * kQTiles) {
+    if (warp >= G::kSoftmaxWarps) {
     // The last warpgroup (producer, MMA and two idle warps) hands registers back in one instruction.
     if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
     if (warp == kProducerWarp) {
@@ -315,11 +331,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     } else {
         // ------------------------------------------------------------------ softmax / correction / epilogue
         if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
-        const int q = warp >> 2;                       // which Q tile this warpgroup owns
-        const int r_in_tile = tid & 127;               // row inside the tile = TMEM lane
+        constexpr int kSplit = G::kSplit, kColsS = G::kColsS, kColsO = G::kColsO;
+        const int q = warp / (4 * kSplit);             // which Q tile this thread works on
+        const int half = (warp >> 2) % kSplit;         // which half of the columns
+        const int r_in_tile = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
+        const int tile_bar = 1 + q;                    // named barrier of the threads that share the tile
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + G::kTmemS + 128 * q;
-        const uint32_t t_o = tmem + lane_base + G::kTmemO + 128 * q;
+        const uint32_t t_s = tmem + lane_base + G::kTmemS + 128 * q + half * kColsS;
+        const uint32_t t_p = tmem + lane_base + G::kTmemS + 128 * q + half * (kColsS / 2);
+        const uint32_t t_o = tmem + lane_base + G::kTmemO + 128 * q + half * kColsO;
+        float* xchg_mine = &bar->xchg[q][half][r_in_tile];
+        const float* xchg_other = &bar->xchg[q][half ^ (kSplit - 1)][r_in_tile];
         const float scale_log2 = p.scale_log2;
         const int N = p.sched.N;
         uint32_t s_phase = 0, o_phase = 0;
@@ -332,27 +354,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int tile_row0 = w.row0 + q * kBlockM;
             const int row = tile_row0 + r_in_tile;
             float m_ref = -INFINITY;   // the max the exponents are taken against (log2 units)
-            float l = 0.f;             // running sum of the probabilities
+            float l = 0.f;             // running sum of this thread's probabilities
             bool first = true;
             for (int s = 0; s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
                 if (j >= hi_mine) continue;
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS));
-                if (!ok) break;
+                const bool got_s = ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS);
                 s_phase ^= 1u;
                 ptx::tc_fence_after();
 
-                uint32_t sv[kBlockN / 32][32];
+                uint32_t sv[kColsS / 32][32];
 #pragma unroll
-                for (int c = 0; c < kBlockN / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
+                for (int c = 0; c < kColsS / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
                 ptx::tmem_wait_ld();
 
-                const int col0 = j * kBlockN;
-                const bool masked = (col0 + kBlockN > N) || (p.sched.causal && (col0 + kBlockN - 1 > tile_row0));
+                const int col0 = j * kBlockN + half * kColsS;  // key index of this thread's first column
+                const bool masked = (j * kBlockN + kBlockN > N) || (p.sched.causal && (j * kBlockN + kBlockN - 1 > tile_row0));
                 if (masked) {
                     const int limit = p.sched.causal ? (row < N - 1 ? row : N - 1) : N - 1;  // last visible key
 #pragma unroll
-                    for (int c = 0; c < kBlockN / 32; ++c)
+                    for (int c = 0; c < kColsS / 32; ++c)
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (col0 + c * 32 + i > limit) sv[c][i] = 0xff800000u;  // -inf
@@ -360,7 +381,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < kBlockN / 32; ++c)
+                for (int c = 0; c < kColsS / 32; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         mx0 = ptx::max3(mx0, __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
@@ -368,7 +389,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         mx2 = ptx::max3(mx2, __uint_as_float(sv[c][i + 4]), __uint_as_float(sv[c][i + 5]));
                         mx3 = ptx::max3(mx3, __uint_as_float(sv[c][i + 6]), __uint_as_float(sv[c][i + 7]));
                     }
-                const float m_cand = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2);
+                float row_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                if (kSplit == 2) {
+                    // The two threads of a row swap their maxima.  The barrier also orders this step's S loads
+                    // of both before either writes P over S's columns, and carries the give-up decision to
+                    // all threads of the tile at once.  (The buffer is free again by the next step: the next
+                    // S exists only after every thread of the tile has arrived on p_full, i.e. has read it.)
+                    *xchg_mine = row_max;
+                    ok = ptx::bar_red_and(tile_bar, G::kTileThreads, got_s);
+                    if (!ok) break;
+                    row_max = fmaxf(row_max, *xchg_other);
+                } else {
+                    ok = ptx::warp_all(got_s);
+                    if (!ok) break;
+                }
+                const float m_cand = fmaxf(m_ref, row_max * scale_log2);
                 const bool need = (m_cand - m_ref) > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
                     float alpha = 1.f;
@@ -380,7 +415,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!first) {
                         // S_q is complete, so every product issued before it, O_q's last update included, is too.
 #pragma unroll 1
-                        for (int c = 0; c < kD / 16; ++c) {
+                        for (int c = 0; c < kColsO / 16; ++c) {
                             uint32_t ov[16];
                             ptx::tmem_ld16(t_o + c * 16, ov);
                             ptx::tmem_wait_ld();
@@ -395,7 +430,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const ptx::f32x2 neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
                 ptx::f32x2 l01 = ptx::pack_f32x2(0.f, 0.f), l23 = ptx::pack_f32x2(0.f, 0.f);
 #pragma unroll
-                for (int c = 0; c < kBlockN / 32; ++c) {
+                for (int c = 0; c < kColsS / 32; ++c) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         uint32_t pk[8];
@@ -417,7 +452,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
                             pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
                         }
-                        ptx::tmem_st8(t_s + c * 16 + h * 8, pk);
+                        ptx::tmem_st8(t_p + c * 16 + h * 8, pk);
                     }
                 }
                 float l0, l1, l2, l3;
@@ -431,14 +466,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             if (!ok) break;
             // ---- epilogue: O_q / l -> 16 bit -> global
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bar->o_full[q], o_phase, abort_flag, kSiteSoftmaxO));
-            if (!ok) break;
+            const bool got_o = ptx::mbar_wait(&bar->o_full[q], o_phase, abort_flag, kSiteSoftmaxO);
             o_phase ^= 1u;
             ptx::tc_fence_after();
+            if (kSplit == 2) {
+                *xchg_mine = l;
+                ok = ptx::bar_red_and(tile_bar, G::kTileThreads, got_o);
+                if (!ok) break;
+                l += *xchg_other;
+            } else {
+                ok = ptx::warp_all(got_o);
+                if (!ok) break;
+            }
             const float inv_l = 1.f / l;
-            uint4* o_row = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.o) + ((size_t)w.bh * N + row) * (size_t)(kD * 2));
+            uint4* o_row = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.o) + ((size_t)w.bh * N + row) * (size_t)(kD * 2) +
+                                                    (size_t)half * (kColsO * 2));
 #pragma unroll
-            for (int c = 0; c < kD / 32; ++c) {
+            for (int c = 0; c < kColsO / 32; ++c) {
                 uint32_t ov[32];
                 ptx::tmem_ld32(t_o + c * 32, ov);
                 ptx::tmem_wait_ld();
@@ -453,9 +497,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             }
             ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
+            // The other thread of the row has read this thread's partial sum before the buffer holds a maximum again.
+            if (kSplit == 2) ptx::bar_sync(tile_bar, G::kTileThreads);
         }
     }
-
 
     ptx::tc_fence_before();
     __syncthreads();
