@@ -141,6 +141,13 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
  */
 int attn_device_status(int* code);
 
+/*
+ * Waits for the current device and returns the SM clock cycles that the first CTA of the most recent
+ * attention kernel spent in its loop over work items (a measuring aid: cycles / elapsed time is the
+ * SM clock the kernel really ran at, which on a power-capped GPU is not the nominal one).
+ */
+int attn_last_kernel_cycles(unsigned long long* cycles);
+
 const char* attn_status_string(int status);
 const char* attn_last_error(void);
 

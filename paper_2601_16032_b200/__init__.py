@@ -8,6 +8,6 @@ from .binding import (  # noqa: F401
     CYCLIC, SAWTOOTH, F16, BF16, TILE_FASTEST, HEAD_FASTEST,
     AttnError, Opts, Plan, TraceEntry,
     attn_fwd, attn_fwd_ex, attn_fwd_host, attn_query_plan, attn_schedule_trace,
-    attn_device_status, attn_status_string, attn_last_error, library_path, load_library,
+    attn_device_status, attn_last_kernel_cycles, attn_status_string, attn_last_error, library_path, load_library,
     forward,
 )

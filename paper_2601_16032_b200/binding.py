@@ -67,6 +67,8 @@ def load_library():
     lib.attn_schedule_trace.argtypes = shape + [ci, ci, ci, ctypes.POINTER(Opts), ci, ctypes.POINTER(TraceEntry),
                                                 ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     lib.attn_device_status.argtypes = [ctypes.POINTER(ci)]
+    lib.attn_last_kernel_cycles.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
+    lib.attn_last_kernel_cycles.restype = ci
     for name in ("attn_fwd", "attn_fwd_ex", "attn_fwd_host", "attn_query_plan", "attn_schedule_trace", "attn_device_status"):
         getattr(lib, name).restype = ci
     lib.attn_status_string.argtypes = [ci]
@@ -134,6 +136,13 @@ def attn_device_status() -> int:
     code = ctypes.c_int(0)
     _check(load_library().attn_device_status(ctypes.byref(code)))
     return code.value
+
+
+def attn_last_kernel_cycles() -> int:
+    """Synchronises the device; SM cycles the first CTA of the most recent kernel spent on its work items."""
+    c = ctypes.c_ulonglong(0)
+    _check(load_library().attn_last_kernel_cycles(ctypes.byref(c)))
+    return int(c.value)
 
 
 def forward(q, k, v, causal: bool = False, scan_order: int = SAWTOOTH, scale: Optional[float] = None,

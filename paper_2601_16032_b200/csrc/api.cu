@@ -25,6 +25,7 @@ int fail(int status, const char* fmt, ...) {
 }
 
 __device__ int g_status_word = 0;
+__device__ unsigned long long g_cycles = 0;
 
 constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
 
@@ -272,6 +273,8 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o, int B, int
     kp.o = o;
     rc = (int)cudaGetSymbolAddress((void**)&kp.status, g_status_word);
     if (rc != 0) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress failed (%d)", rc); }
+    rc = (int)cudaGetSymbolAddress((void**)&kp.cycles, g_cycles);
+    if (rc != 0) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress failed (%d)", rc); }
 
     CUtensorMap tq, tk, tv;
     if ((rc = make_map(&tq, q, B * H, N, d, kBlockM, dtype))) return rc;
@@ -311,6 +314,15 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
         cudaGetLastError();
         return fail(ATTN_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
     }
+    return ATTN_OK;
+}
+
+int attn_last_kernel_cycles(unsigned long long* cycles) {
+    if (!cycles) return fail(ATTN_ERR_INVALID_ARG, "cycles is null");
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e)); }
+    e = cudaMemcpyFromSymbol(cycles, g_cycles, sizeof(unsigned long long));
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "reading the cycle count: %s", cudaGetErrorString(e)); }
     return ATTN_OK;
 }
 

@@ -29,6 +29,7 @@ struct KernelParams {
     int l2_policy;        // 1: K/V loads evict_last, Q loads evict_first
     void* o;              // [B, H, N, d] output
     int* status;          // device status word (0 = fine)
+    unsigned long long* cycles;  // CTA 0 leaves the SM cycles its MMA loop took here
 };
 
 constexpr int kMaxStages = 16;
@@ -50,7 +51,7 @@ enum WaitSite {
 struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
     uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
@@ -67,6 +68,10 @@ struct Geometry {
     static constexpr int kSplit = SAW_THREADS_PER_ROW;      // threads per query row (1 or 2)
     static constexpr int kColsS = kBlockN / kSplit;         // S columns a softmax thread owns
     static constexpr int kColsO = kD / kSplit;              // O columns a softmax thread owns
+    // P reaches the MMA warp in two parts: a thread announces its first kEarlyGroups groups of 16
+    // probabilities (one K step of the P.V product each) while it still computes the rest.
+    static constexpr int kGroups = kColsS / 16;
+    static constexpr int kEarlyGroups = kGroups >= 4 ? (kGroups * 3) / 4 : kGroups / 2;
     static constexpr int kSoftmaxWarps = kQTiles * kSplit * 4;
     static constexpr int kTileThreads = 128 * kSplit;       // threads that share one Q tile (one named barrier)
     static constexpr int kThreads = kSoftmaxWarps * 32 + 128;  // plus one warpgroup: producer, MMA, two idle warps
@@ -133,6 +138,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         for (int q = 0; q < 2; ++q) {
             ptx::mbar_init(&bar->s_full[q], 1);
+            ptx::mbar_init(&bar->p_early[q], G::kTileThreads);
             ptx::mbar_init(&bar->p_full[q], G::kTileThreads);
             ptx::mbar_init(&bar->o_full[q], 1);
         }
@@ -250,20 +256,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             b0 + (uint64_t)((c * G::kKVChunkBytes + kk * 32) >> 4), idesc_qk, i != 0);
             }
         };
-        auto issue_pv = [&](int q, int slot, uint32_t accumulate) {
+        // The K steps of O_q += P_q V_j whose 16 probabilities belong to the early part of P (late = 0) or
+        // to the rest (late = 1); a sum, so the order of the steps is free.
+        auto issue_pv = [&](int q, int slot, uint32_t accumulate, int late) {
             const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
             const uint32_t d_tmem = tmem + G::kTmemO + 128 * q;
             const uint32_t a_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk) {
+                if (((kk % G::kGroups) >= G::kEarlyGroups) != (late != 0)) continue;
                 ptx::mma_ts(d_tmem, a_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
-                            accumulate | (kk != 0));
+                            accumulate | (late != 0) | (kk != 0));
             }
         };
 
         // One elected lane runs the whole loop: every wait, issue and commit below is a single
         // thread's, with no warp votes or re-convergence between the MMA batches.
         if (ptx::elect_one()) {
+            const long long clk_begin = clock64();
             int it = 0;
             for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
                 const WorkItem w = decode_work(p.sched, k, it);
@@ -299,10 +309,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int q = 0; q < kQTiles; ++q) {
                         if (j < w.hi_q[q]) {
+                            if (!ptx::mbar_wait(&bar->p_early[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            issue_pv(q, slot_v, pv_started[q], 0);
                             if (!ptx::mbar_wait(&bar->p_full[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
                             p_phase[q] ^= 1u;
                             ptx::tc_fence_after();
-                            issue_pv(q, slot_v, pv_started[q]);
+                            issue_pv(q, slot_v, pv_started[q], 1);
                             pv_started[q] = 1;
                         }
                         if (has_next && j_next < w.hi_q[q]) {
@@ -325,6 +338,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // Nothing of this thread's MMAs may be in flight when TMEM is released.
             ptx::mma_commit(&bar->drain);
             drain_wait(&bar->drain, 0);
+            if (blockIdx.x == 0) *p.cycles = (unsigned long long)(clock64() - clk_begin);
         }
         __syncwarp();
     }
@@ -453,6 +467,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
                         }
                         ptx::tmem_st8(t_p + c * 16 + h * 8, pk);
+                        if (c * 2 + h == G::kEarlyGroups - 1) {
+                            ptx::tmem_wait_st();
+                            ptx::tc_fence_before();
+                            ptx::mbar_arrive(&bar->p_early[q]);
+                        }
                     }
                 }
                 float l0, l1, l2, l3;
