@@ -326,6 +326,16 @@ int attn_last_kernel_cycles(unsigned long long* cycles) {
     return ATTN_OK;
 }
 
+#ifdef SAW_PROFILE
+/* Profiling builds only: copies the per-CTA phase table (256 x 32 cycle counts) to `out` after a device sync. */
+int attn_debug_profile(unsigned long long* out) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(out, sawtooth::g_profile, sizeof(unsigned long long) * 256 * 32);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "reading the profile table: %s", cudaGetErrorString(e)); }
+    return ATTN_OK;
+}
+#endif
+
 int attn_device_status(int* code) {
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e)); }
