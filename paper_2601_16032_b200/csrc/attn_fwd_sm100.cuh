@@ -2,17 +2,18 @@
 // S, P and O in tensor memory, one softmax thread per query row.
 //
 // One CTA handles work items of kQTiles x 128 query rows (Algorithm 1's resident Q tile).  Warp roles:
-//   warps [0, 8*kQTiles)   softmax: two warpgroups per Q tile; row r of the tile (TMEM lane r) is shared
-//                          by two threads, one per half of the K/V tile's columns.  Each reads its half
-//                          of S from TMEM, the two exchange their row maxima through shared memory,
-//                          keep the running max and a partial sum, write P back to TMEM as 16-bit
-//                          pairs, rescale their half of O's columns when the max moved, and at the end
-//                          of the item normalise and store their half of the O row.
-//   warp 8*kQTiles         producer: one elected lane issues the TMA loads (Q tiles, then K_j, V_j in
+//   the softmax warps      one warpgroup per Q tile, thread r owning row r (TMEM lane r), or, built with
+//                          SAW_THREADS_PER_ROW=2, two warpgroups per tile whose threads split a row's
+//                          columns and exchange their row maxima through shared memory.  A thread reads
+//                          its part of S from TMEM, keeps the running max and a (partial) sum, writes P
+//                          back to TMEM as 16-bit pairs, rescales its part of O when the max moved, and
+//                          at the end of the item normalises and stores its part of the O row.
+//   the next warp          producer: one elected lane issues the TMA loads (Q tiles, then K_j, V_j in
 //                          the scan order of the item) into a ring of shared-memory slots.
-//   warp 8*kQTiles + 1     MMA: one elected lane issues S_q = Q_q K_j^T and O_q += P_q V_j and commits
-//                          them to mbarriers; the warp also owns the TMEM allocation.
-//   two more warps         idle; they complete the warpgroup whose registers go to the softmax threads.
+//   the next kQTiles warps MMA, one warp per Q tile q: one elected lane issues S_q = Q_q K_j^T and
+//                          O_q += P_q V_j and commits them to mbarriers; the first of them also owns
+//                          the TMEM allocation.
+//   the remaining warp(s)  idle; they complete the warpgroup whose registers go to the softmax threads.
 // With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
 // Four softmax warps per scheduler (two threads per row) keep the MUFU busy: one warp alone can start
 // an exponential only every other MUFU slot.
@@ -21,6 +22,19 @@
 #include "schedule.h"
 
 namespace sawtooth {
+
+// Optional in-kernel clock stamps (build with -DSAW_PROFILE): one thread of each role of every CTA adds up
+// the SM cycles it spends in each phase; the host reads the table with attn_debug_profile().
+#ifdef SAW_PROFILE
+__device__ unsigned long long g_profile[256][32];
+#define SAW_PROF_DECL long long prof_t = clock64(); long long prof_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define SAW_PROF(slot) do { const long long prof_n = clock64(); prof_acc[slot] += prof_n - prof_t; prof_t = prof_n; } while (0)
+#define SAW_PROF_WRITE(base, cond) do { if (cond) { for (int prof_i = 0; prof_i < 12; ++prof_i) g_profile[blockIdx.x & 255][(base) + prof_i] = (unsigned long long)prof_acc[prof_i]; } } while (0)
+#else
+#define SAW_PROF_DECL do { } while (0)
+#define SAW_PROF(slot) do { } while (0)
+#define SAW_PROF_WRITE(base, cond) do { } while (0)
+#endif
 
 struct KernelParams {
     SchedParams sched;
@@ -34,10 +48,10 @@ struct KernelParams {
 
 constexpr int kMaxStages = 16;
 #ifndef SAW_THREADS_PER_ROW
-#define SAW_THREADS_PER_ROW 2
+#define SAW_THREADS_PER_ROW 1
 #endif
 #ifndef SAW_EXP_POLY_OF_4
-#define SAW_EXP_POLY_OF_4 0
+#define SAW_EXP_POLY_OF_4 1
 #endif
 constexpr int kExpPolyOf4 = SAW_EXP_POLY_OF_4;  // of every four pairs of exponentials, how many avoid the MUFU
 constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the row max grew by more (log2 units)
@@ -52,7 +66,7 @@ struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
     uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
-    uint64_t drain;
+    uint64_t drain[2];
     uint32_t tmem_base;
     int abort_flag;
     float xchg[2][2][128];  // [Q tile][column half][row]: row maxima, and the partial row sums at the end of an item
@@ -131,10 +145,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (tid == 0) {
         ptx::mbar_init(&bar->q_full, 1);
-        ptx::mbar_init(&bar->q_empty, 1);
+        ptx::mbar_init(&bar->q_empty, kQTiles);
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(&bar->kv_full[s], 1);
-            ptx::mbar_init(&bar->kv_empty[s], 1);
+            ptx::mbar_init(&bar->kv_empty[s], kQTiles);
         }
         for (int q = 0; q < 2; ++q) {
             ptx::mbar_init(&bar->s_full[q], 1);
@@ -142,7 +156,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ptx::mbar_init(&bar->p_full[q], G::kTileThreads);
             ptx::mbar_init(&bar->o_full[q], 1);
         }
-        ptx::mbar_init(&bar->drain, 1);
+        ptx::mbar_init(&bar->drain[0], 1);
+        ptx::mbar_init(&bar->drain[1], 1);
         bar->abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -231,73 +246,74 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
         }
         __syncwarp();
-    } else if (warp == kMmaWarp) {
+    } else if (warp < kMmaWarp + kQTiles) {
         // ------------------------------------------------------------------ MMA issue
+        // One warp per Q tile, one elected lane each: the products of the two tiles are independent, so
+        // a lane that waits for its tile's P does not hold up the other tile's products.  Both lanes walk
+        // the same K/V ring; a slot, and the Q buffer, are free again once both have committed.
+        const int q = warp - kMmaWarp;
         constexpr uint32_t idesc_qk = ptx::instr_desc_f16(kBf16, 0, kBlockM, kBlockN);
         constexpr uint32_t idesc_pv = ptx::instr_desc_f16(kBf16, 1, kBlockM, kD);
         const uint32_t q_base = ptx::smem_u32(q_smem);
         const uint32_t kv_base = ptx::smem_u32(kv_smem);
         Ring ring;
-        uint32_t p_phase[2] = {0, 0};
+        uint32_t p_phase = 0;
         bool ok = true;
 
         // Descriptors differ from a base only in the 16-byte-granular address field (the low bits).
-        const uint64_t q_desc0 = ptx::smem_desc_sw128(q_base, 16, 1024);
+        const uint64_t q_desc = ptx::smem_desc_sw128(q_base, 16, 1024) + (uint64_t)((q * G::kQTileBytes) >> 4);
         const uint64_t k_desc0 = ptx::smem_desc_sw128(kv_base, 16, 1024);
         const uint64_t v_desc0 = ptx::smem_desc_sw128(kv_base, G::kKVChunkBytes, 1024);
-        auto issue_qk = [&](int q, int slot) {
-            const uint64_t a0 = q_desc0 + (uint64_t)((q * G::kQTileBytes) >> 4);
+        const uint32_t s_tmem = tmem + G::kTmemS + 128 * q;
+        const uint32_t o_tmem = tmem + G::kTmemO + 128 * q;
+        auto issue_qk = [&](int slot) {
             const uint64_t b0 = k_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
-            const uint32_t d_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
             for (int i = 0; i < G::kChunks * 4; ++i) {
                 const int c = i >> 2, kk = i & 3;
-                ptx::mma_ss(d_tmem, a0 + (uint64_t)((c * G::kQChunkBytes + kk * 32) >> 4),
+                ptx::mma_ss(s_tmem, q_desc + (uint64_t)((c * G::kQChunkBytes + kk * 32) >> 4),
                             b0 + (uint64_t)((c * G::kKVChunkBytes + kk * 32) >> 4), idesc_qk, i != 0);
             }
         };
         // The K steps of O_q += P_q V_j whose 16 probabilities belong to the early part of P (late = 0) or
         // to the rest (late = 1); a sum, so the order of the steps is free.
-        auto issue_pv = [&](int q, int slot, uint32_t accumulate, int late) {
+        auto issue_pv = [&](int slot, uint32_t accumulate, int late) {
             const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
-            const uint32_t d_tmem = tmem + G::kTmemO + 128 * q;
-            const uint32_t a_tmem = tmem + G::kTmemS + 128 * q;
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk) {
                 if (((kk % G::kGroups) >= G::kEarlyGroups) != (late != 0)) continue;
-                ptx::mma_ts(d_tmem, a_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
+                ptx::mma_ts(o_tmem, s_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
                             accumulate | (late != 0) | (kk != 0));
             }
         };
 
-        // One elected lane runs the whole loop: every wait, issue and commit below is a single
+        // The elected lane runs the whole loop: every wait, issue and commit below is a single
         // thread's, with no warp votes or re-convergence between the MMA batches.
         if (ptx::elect_one()) {
             const long long clk_begin = clock64();
+            SAW_PROF_DECL;
             int it = 0;
             for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
                 const WorkItem w = decode_work(p.sched, k, it);
+                const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
+                SAW_PROF(0);
                 if (!ptx::mbar_wait(&bar->q_full, it & 1, abort_flag, kSiteMmaQ)) { ok = false; break; }
+                SAW_PROF(1);
                 // K tile of step 0
                 const int slot_k = ring.slot;
                 if (!ptx::mbar_wait(&bar->kv_full[slot_k], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                 ring.advance(stages);
                 ptx::tc_fence_after();
-                {
-                    const int j0 = kv_tile_at(w, 0);
-#pragma unroll
-                    for (int q = 0; q < kQTiles; ++q) {
-                        if (j0 < w.hi_q[q]) { issue_qk(q, slot_k); ptx::mma_commit(&bar->s_full[q]); }
-                    }
-                    ptx::mma_commit(&bar->kv_empty[slot_k]);
-                    if (w.hi == 1) ptx::mma_commit(&bar->q_empty);
-                }
-                uint32_t pv_started[2] = {0, 0};
+                if (kv_tile_at(w, 0) < hi_mine) { issue_qk(slot_k); ptx::mma_commit(&bar->s_full[q]); }
+                ptx::mma_commit(&bar->kv_empty[slot_k]);
+                if (w.hi == 1) ptx::mma_commit(&bar->q_empty);
+                uint32_t pv_started = 0;
                 for (int s = 0; ok && s < w.hi; ++s) {
                     const int j = kv_tile_at(w, s);
                     const bool has_next = s + 1 < w.hi;
                     const int j_next = has_next ? kv_tile_at(w, s + 1) : 0;
                     const int slot_v = ring.slot;
+                    SAW_PROF(0);
                     if (!ptx::mbar_wait(&bar->kv_full[slot_v], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                     ring.advance(stages);
                     int slot_kn = 0;
@@ -306,39 +322,43 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (!ptx::mbar_wait(&bar->kv_full[slot_kn], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                         ring.advance(stages);
                     }
-#pragma unroll
-                    for (int q = 0; q < kQTiles; ++q) {
-                        if (j < w.hi_q[q]) {
-                            if (!ptx::mbar_wait(&bar->p_early[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
-                            ptx::tc_fence_after();
-                            issue_pv(q, slot_v, pv_started[q], 0);
-                            if (!ptx::mbar_wait(&bar->p_full[q], p_phase[q], abort_flag, kSiteMmaP)) { ok = false; break; }
-                            p_phase[q] ^= 1u;
-                            ptx::tc_fence_after();
-                            issue_pv(q, slot_v, pv_started[q], 1);
-                            pv_started[q] = 1;
-                        }
-                        if (has_next && j_next < w.hi_q[q]) {
-                            issue_qk(q, slot_kn);
-                            ptx::mma_commit(&bar->s_full[q]);
-                        }
+                    SAW_PROF(2);
+                    if (j < hi_mine) {
+                        if (!ptx::mbar_wait(&bar->p_early[q], p_phase, abort_flag, kSiteMmaP)) { ok = false; break; }
+                        SAW_PROF(3);
+                        ptx::tc_fence_after();
+                        issue_pv(slot_v, pv_started, 0);
+                        SAW_PROF(4);
+                        if (!ptx::mbar_wait(&bar->p_full[q], p_phase, abort_flag, kSiteMmaP)) { ok = false; break; }
+                        SAW_PROF(5);
+                        p_phase ^= 1u;
+                        ptx::tc_fence_after();
+                        issue_pv(slot_v, pv_started, 1);
+                        pv_started = 1;
+                        SAW_PROF(6);
                     }
-                    if (!ok) break;
+                    if (has_next && j_next < hi_mine) {
+                        ptx::tc_fence_after();
+                        issue_qk(slot_kn);
+                        ptx::mma_commit(&bar->s_full[q]);
+                        SAW_PROF(7);
+                    }
+                    // Every lane commits every slot, used by its tile or not: the slot's count is the number of lanes.
                     ptx::mma_commit(&bar->kv_empty[slot_v]);
                     if (has_next) {
                         ptx::mma_commit(&bar->kv_empty[slot_kn]);
-                        if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S products are issued
+                        if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S product is issued
                     }
+                    SAW_PROF(8);
                 }
                 if (!ok) break;
-#pragma unroll
-                for (int q = 0; q < kQTiles; ++q)
-                    if (w.hi_q[q] > 0) ptx::mma_commit(&bar->o_full[q]);
+                if (hi_mine > 0) ptx::mma_commit(&bar->o_full[q]);
             }
             // Nothing of this thread's MMAs may be in flight when TMEM is released.
-            ptx::mma_commit(&bar->drain);
-            drain_wait(&bar->drain, 0);
-            if (blockIdx.x == 0) *p.cycles = (unsigned long long)(clock64() - clk_begin);
+            ptx::mma_commit(&bar->drain[q]);
+            drain_wait(&bar->drain[q], 0);
+            if (blockIdx.x == 0 && q == 0) *p.cycles = (unsigned long long)(clock64() - clk_begin);
+            SAW_PROF_WRITE(0, q == 0);
         }
         __syncwarp();
     }
@@ -361,6 +381,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t s_phase = 0, o_phase = 0;
         bool ok = true;
         int it = 0;
+        SAW_PROF_DECL;
         for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
             const WorkItem w = decode_work(p.sched, k, it);
             const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
@@ -373,14 +394,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int s = 0; s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
                 if (j >= hi_mine) continue;
+                SAW_PROF(0);
                 const bool got_s = ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS);
                 s_phase ^= 1u;
                 ptx::tc_fence_after();
+                SAW_PROF(1);
 
                 uint32_t sv[kColsS / 32][32];
 #pragma unroll
                 for (int c = 0; c < kColsS / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
                 ptx::tmem_wait_ld();
+                SAW_PROF(2);
 
                 const int col0 = j * kBlockN + half * kColsS;  // key index of this thread's first column
                 const bool masked = (j * kBlockN + kBlockN > N) || (p.sched.causal && (j * kBlockN + kBlockN - 1 > tile_row0));
@@ -393,17 +417,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             if (col0 + c * 32 + i > limit) sv[c][i] = 0xff800000u;  // -inf
                 }
 
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                // Eight independent chains of three-input maxima, then a tree.
+                float mx[8];
 #pragma unroll
-                for (int c = 0; c < kColsS / 32; ++c)
+                for (int i = 0; i < 8; ++i) mx[i] = ptx::max3(__uint_as_float(sv[0][3 * i]), __uint_as_float(sv[0][3 * i + 1]), __uint_as_float(sv[0][3 * i + 2]));
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        mx0 = ptx::max3(mx0, __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
-                        mx1 = ptx::max3(mx1, __uint_as_float(sv[c][i + 2]), __uint_as_float(sv[c][i + 3]));
-                        mx2 = ptx::max3(mx2, __uint_as_float(sv[c][i + 4]), __uint_as_float(sv[c][i + 5]));
-                        mx3 = ptx::max3(mx3, __uint_as_float(sv[c][i + 6]), __uint_as_float(sv[c][i + 7]));
-                    }
-                float row_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                for (int i = 0; i < 4; ++i) mx[i] = ptx::max3(mx[i], __uint_as_float(sv[0][24 + 2 * i]), __uint_as_float(sv[0][25 + 2 * i]));
+#pragma unroll
+                for (int c = 1; c < kColsS / 32; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2)
+                        mx[(i >> 1) & 7] = ptx::max3(mx[(i >> 1) & 7], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
+                float row_max = fmaxf(ptx::max3(mx[0], mx[1], mx[2]), fmaxf(ptx::max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                SAW_PROF(3);
                 if (kSplit == 2) {
                     // The two threads of a row swap their maxima.  The barrier also orders this step's S loads
                     // of both before either writes P over S's columns, and carries the give-up decision to
@@ -417,6 +443,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ok = ptx::warp_all(got_s);
                     if (!ok) break;
                 }
+                SAW_PROF(4);
                 const float m_cand = fmaxf(m_ref, row_max * scale_log2);
                 const bool need = (m_cand - m_ref) > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
@@ -439,41 +466,48 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
+                SAW_PROF(5);
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
                 const ptx::f32x2 scale2 = ptx::pack_f32x2(scale_log2, scale_log2);
                 const ptx::f32x2 neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
                 ptx::f32x2 l01 = ptx::pack_f32x2(0.f, 0.f), l23 = ptx::pack_f32x2(0.f, 0.f);
-#pragma unroll
-                for (int c = 0; c < kColsS / 32; ++c) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4) {
-                            // Four probabilities: x = S * scale * log2(e) - m as two packed FMAs, then 2^x on the MUFU
-                            // or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
-                            const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
-                            const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
-                            float x0, x1, x2, x3, p0, p1, p2, p3;
-                            ptx::unpack_f32x2(xa, x0, x1);
-                            ptx::unpack_f32x2(xb, x2, x3);
-                            if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
-                            else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
-                            if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
-                            else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
-                            l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
-                            l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
-                            pk[i / 2] = ptx::pack2<kBf16>(p0, p1);
-                            pk[i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
-                        }
-                        ptx::tmem_st8(t_p + c * 16 + h * 8, pk);
-                        if (c * 2 + h == G::kEarlyGroups - 1) {
-                            ptx::tmem_wait_st();
-                            ptx::tc_fence_before();
-                            ptx::mbar_arrive(&bar->p_early[q]);
-                        }
+                // Groups of 16 probabilities (eight packed registers, one TMEM store each).  The store of a
+                // group is issued after the exponentials of the next group, so that it never waits in the
+                // instruction stream for MUFU results that are still in flight.
+                uint32_t pk[G::kGroups][8];
+                auto finish_group = [&](int g) {
+                    ptx::tmem_st8(t_p + g * 8, pk[g]);
+                    if (g == G::kEarlyGroups - 1) {
+                        ptx::tmem_wait_st();
+                        ptx::tc_fence_before();
+                        ptx::mbar_arrive(&bar->p_early[q]);
+                        SAW_PROF(6);
                     }
+                };
+#pragma unroll
+                for (int g = 0; g < G::kGroups; ++g) {
+                    const int c = g >> 1, h = g & 1;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        // Four probabilities: x = S * scale * log2(e) - m as two packed FMAs, then 2^x on the MUFU
+                        // or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
+                        const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
+                        const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
+                        float x0, x1, x2, x3, p0, p1, p2, p3;
+                        ptx::unpack_f32x2(xa, x0, x1);
+                        ptx::unpack_f32x2(xb, x2, x3);
+                        if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
+                        else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
+                        if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
+                        else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
+                        l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
+                        l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
+                        pk[g][i / 2] = ptx::pack2<kBf16>(p0, p1);
+                        pk[g][i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
+                    }
+                    if (g > 0) finish_group(g - 1);
                 }
+                finish_group(G::kGroups - 1);
                 float l0, l1, l2, l3;
                 ptx::unpack_f32x2(l01, l0, l1);
                 ptx::unpack_f32x2(l23, l2, l3);
@@ -481,6 +515,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(&bar->p_full[q]);
+                SAW_PROF(7);
                 first = false;
             }
             if (!ok) break;
@@ -518,7 +553,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
             // The other thread of the row has read this thread's partial sum before the buffer holds a maximum again.
             if (kSplit == 2) ptx::bar_sync(tile_bar, G::kTileThreads);
+            SAW_PROF(8);
         }
+        SAW_PROF_WRITE(12, q == 0 && half == 0 && r_in_tile == 0);
     }
 
     ptx::tc_fence_before();
