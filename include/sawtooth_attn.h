@@ -108,6 +108,26 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o,
                 int dtype, void* stream, const attn_fwd_opts* opts);
 
 /*
+ * The same forward pass with a DYNAMIC tile schedule in place of Algorithm 2's static grid-stride walk (the paper's
+ * persistent loop hands CTA c the items c, c+G, ...; under the causal mask those differ in length by up to the whole
+ * sequence, and CTAs that drew short ones idle at the end).  Here every persistent CTA claims its next work item from
+ * a counter in `scratch`, in index order, which under the causal mask runs from the longest Q block of a head to the
+ * shortest.  Algorithm 4's alternation still follows the CTA's own count of items, so which items a CTA scans
+ * backward depends on the race for the counter: results are reproducible bit for bit in the cyclic order only.
+ *
+ * scratch: DEVICE memory owned by the caller, 4-byte aligned, at least attn_dynamic_scratch_bytes(plan.grid) bytes
+ * (plan from attn_query_plan; ATTN_DYNAMIC_SCRATCH_HEADER + 4 bytes per CTA).  The call clears it on `stream` before
+ * the kernel; afterwards int[0] holds the number of claims made and int[64 + c] the number of items CTA c handled.
+ * Two calls that share one scratch buffer must not overlap on the GPU.  launch_mode must be 0.
+ */
+#define ATTN_DYNAMIC_SCRATCH_HEADER 256
+size_t attn_dynamic_scratch_bytes(int ctas);
+int attn_fwd_dynamic(const void* q, const void* k, const void* v, void* o,
+                     int B, int H, int N, int d, float scale, int causal, int scan_order,
+                     int dtype, void* stream, const attn_fwd_opts* opts,
+                     void* scratch, size_t scratch_bytes);
+
+/*
  * Same computation for HOST buffers: copies q, k, v (host, ideally pinned) into the caller's device
  * staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host,
  * all enqueued on `stream`.  Each buffer holds B*H*N*d 16-bit elements.  Returns without waiting:

@@ -62,6 +62,10 @@ def load_library():
     shape = [ci, ci, ci, ci]
     lib.attn_fwd.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp]
     lib.attn_fwd_ex.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts)]
+    lib.attn_fwd_dynamic.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts), vp, ctypes.c_size_t]
+    lib.attn_fwd_dynamic.restype = ci
+    lib.attn_dynamic_scratch_bytes.argtypes = [ci]
+    lib.attn_dynamic_scratch_bytes.restype = ctypes.c_size_t
     lib.attn_fwd_host.argtypes = [vp] * 8 + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts)]
     lib.attn_query_plan.argtypes = shape + [ci, ci, ctypes.POINTER(Opts), ci, ctypes.POINTER(Plan)]
     lib.attn_schedule_trace.argtypes = shape + [ci, ci, ci, ctypes.POINTER(Opts), ci, ctypes.POINTER(TraceEntry),
@@ -105,6 +109,18 @@ def attn_fwd(q: int, k: int, v: int, o: int, B: int, H: int, N: int, d: int, sca
 def attn_fwd_ex(q: int, k: int, v: int, o: int, B: int, H: int, N: int, d: int, scale: float, causal: int,
                 scan_order: int, dtype: int, stream: int = 0, opts: Optional[Opts] = None) -> None:
     _check(load_library().attn_fwd_ex(q, k, v, o, B, H, N, d, scale, int(causal), scan_order, dtype, stream, _opts_ptr(opts)))
+
+
+def attn_dynamic_scratch_bytes(ctas: int) -> int:
+    return int(load_library().attn_dynamic_scratch_bytes(ctas))
+
+
+def attn_fwd_dynamic(q: int, k: int, v: int, o: int, B: int, H: int, N: int, d: int, scale: float, causal: int,
+                     scan_order: int, dtype: int, stream: int = 0, opts: Optional[Opts] = None, scratch: int = 0,
+                     scratch_bytes: int = 0) -> None:
+    """attn_fwd_ex with the dynamic tile schedule; scratch: device address of the caller's counter buffer."""
+    _check(load_library().attn_fwd_dynamic(q, k, v, o, B, H, N, d, scale, int(causal), scan_order, dtype, stream,
+                                           _opts_ptr(opts), scratch, scratch_bytes))
 
 
 def attn_fwd_host(q_host: int, k_host: int, v_host: int, o_host: int, q_dev: int, k_dev: int, v_dev: int, o_dev: int,

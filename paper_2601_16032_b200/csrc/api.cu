@@ -248,8 +248,30 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
     return ATTN_OK;
 }
 
+static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                      int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, int* work_counter, size_t counter_bytes,
+                      int counter_ctas_max);
+
 int attn_fwd_ex(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
                 int scan_order, int dtype, void* stream, const attn_fwd_opts* opts) {
+    return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, nullptr, 0, 0);
+}
+
+size_t attn_dynamic_scratch_bytes(int ctas) { return (size_t)ATTN_DYNAMIC_SCRATCH_HEADER + 4u * (size_t)(ctas > 0 ? ctas : 0); }
+
+int attn_fwd_dynamic(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                     int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, void* scratch, size_t scratch_bytes) {
+    if (!scratch) return fail(ATTN_ERR_INVALID_ARG, "scratch is null");
+    if ((uintptr_t)scratch & 3u) return fail(ATTN_ERR_ALIGNMENT, "scratch must be 4-byte aligned");
+    if (scratch_bytes < (size_t)ATTN_DYNAMIC_SCRATCH_HEADER) return fail(ATTN_ERR_INVALID_ARG, "scratch is smaller than its %d-byte header", ATTN_DYNAMIC_SCRATCH_HEADER);
+    const size_t ctas_max = (scratch_bytes - ATTN_DYNAMIC_SCRATCH_HEADER) / 4;
+    return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, static_cast<int*>(scratch), scratch_bytes,
+                      (int)(ctas_max < 2147483647u ? ctas_max : 2147483647u));
+}
+
+static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                      int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, int* work_counter, size_t counter_bytes,
+                      int counter_ctas_max) {
     if (!q || !k || !v || !o) return fail(ATTN_ERR_INVALID_ARG, "q, k, v and o must be non-null");
     int rc = check_shape(B, H, N, d, causal, dtype);
     if (rc) return rc;
@@ -266,7 +288,11 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o, int B, int
     if (rc) return rc;
 
     KernelParams kp;
-    kp.sched = make_sched(B, H, N, r.q_tiles, r.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, r.head_fastest);
+    // Dynamic schedule: items are claimed in index order, and under the causal mask that order runs from the last
+    // (longest) Q block of a head to the first, so that the short items fill the end of the launch.
+    kp.sched = make_sched(B, H, N, r.q_tiles, r.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, r.head_fastest,
+                          work_counter != nullptr && causal);
+    kp.work_counter = work_counter;
     kp.scale_log2 = scale * 1.4426950408889634f;
     kp.kv_stages = r.stages;
     kp.l2_policy = r.l2_policy;
@@ -283,6 +309,15 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o, int B, int
 
     const int grid = grid_for(kp.sched.n_work, sm_count, r);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (work_counter) {
+        if (r.launch_mode != 0) return fail(ATTN_ERR_INVALID_ARG, "the dynamic schedule needs the persistent launch (launch_mode 0)");
+        if (grid > counter_ctas_max)
+            return fail(ATTN_ERR_INVALID_ARG, "scratch holds counters for %d CTAs, the launch has %d (need %zu bytes)", counter_ctas_max, grid,
+                        (size_t)ATTN_DYNAMIC_SCRATCH_HEADER + 4u * (size_t)grid);
+        (void)counter_bytes;
+        cudaError_t e = cudaMemsetAsync(work_counter, 0, (size_t)ATTN_DYNAMIC_SCRATCH_HEADER + 4u * (size_t)grid, st);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "clearing the scratch: %s", cudaGetErrorString(e)); }
+    }
     return d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st)
                     : launch_tiles<64>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st);
 }

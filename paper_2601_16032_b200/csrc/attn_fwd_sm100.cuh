@@ -44,6 +44,8 @@ struct KernelParams {
     void* o;              // [B, H, N, d] output
     int* status;          // device status word (0 = fine)
     unsigned long long* cycles;  // CTA 0 leaves the SM cycles its MMA loop took here
+    int* work_counter;    // dynamic schedule: [0] next unclaimed work index (zero at launch), [64 + cta] items the CTA
+                          // handled; nullptr: the static grid-stride schedule of Algorithm 2
 };
 
 constexpr int kMaxStages = 16;
@@ -59,7 +61,7 @@ constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the
 // Codes written to the status word: which wait gave up.
 enum WaitSite {
     kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
-    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8
+    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8, kSiteWorkFull = 9, kSiteWorkEmpty = 10
 };
 
 struct __align__(8) Barriers {
@@ -67,6 +69,8 @@ struct __align__(8) Barriers {
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
     uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
     uint64_t drain[2];
+    uint64_t work_full[2], work_empty[2];  // dynamic schedule: two-slot mailbox of claimed work indices
+    long long work_k[2];
     uint32_t tmem_base;
     int abort_flag;
     float xchg[2][2][128];  // [Q tile][column half][row]: row maxima, and the partial row sums at the end of an item
@@ -156,6 +160,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ptx::mbar_init(&bar->p_full[q], G::kTileThreads);
             ptx::mbar_init(&bar->o_full[q], 1);
         }
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&bar->work_full[i], 1);
+            ptx::mbar_init(&bar->work_empty[i], kQTiles + G::kSoftmaxWarps);
+        }
         ptx::mbar_init(&bar->drain[0], 1);
         ptx::mbar_init(&bar->drain[1], 1);
         bar->abort_flag = 0;
@@ -175,8 +183,43 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     ptx::tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
 
-    const long long k_first = blockIdx.x;
-    const long long k_stride = gridDim.x;
+    // Which work item this CTA handles as its iteration `it` (-1: none left).  Static schedule (Algorithm 2):
+    // blockIdx.x + it * gridDim.x.  Dynamic schedule: the producer warp claims the next unclaimed index from a
+    // global counter and passes it to the other roles through a two-slot mailbox in shared memory, so a CTA
+    // that drew short items simply draws more of them; Algorithm 4's parity stays the CTA's own count `it`.
+    const bool dynamic = p.work_counter != nullptr;
+    auto static_work = [&](int it) -> long long {
+        const long long k = (long long)blockIdx.x + (long long)it * gridDim.x;
+        return k < p.sched.n_work ? k : -1;
+    };
+    auto claim_work = [&](int it, bool& ok) -> long long {  // producer warp, all lanes
+        if (!dynamic) return static_work(it);
+        const int slot = it & 1;
+        if (it >= 2) {
+            ok = ptx::warp_all(ptx::mbar_wait(&bar->work_empty[slot], (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag, kSiteWorkEmpty));
+            if (!ok) return -1;
+        }
+        if (ptx::elect_one()) {
+            const long long c = (long long)atomicAdd(p.work_counter, 1);
+            bar->work_k[slot] = c < p.sched.n_work ? c : -1;
+            ptx::mbar_arrive(&bar->work_full[slot]);
+        }
+        __syncwarp();
+        return bar->work_k[slot];
+    };
+    auto take_work = [&](int it, bool& ok, bool whole_warp) -> long long {  // MMA lanes (one thread), softmax warps
+        if (!dynamic) return static_work(it);
+        const int slot = it & 1;
+        if (!ptx::mbar_wait(&bar->work_full[slot], (uint32_t)((it >> 1) & 1), abort_flag, kSiteWorkFull)) { ok = false; return -1; }
+        const long long k = bar->work_k[slot];
+        if (whole_warp) {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&bar->work_empty[slot]);
+        } else {
+            ptx::mbar_arrive(&bar->work_empty[slot]);
+        }
+        return k;
+    };
 
     if (warp >= G::kSoftmaxWarps) {
     // The last warpgroup (producer, MMA and two idle warps) hands registers back in one instruction.
@@ -192,7 +235,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         long long kv_issued = 0;   // K/V tile loads issued so far
         bool ok = true;
         int it = 0;
-        for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+        for (; ok; ++it) {
+            const long long k = claim_work(it, ok);
+            if (!ok || k < 0) break;
             const WorkItem w = decode_work(p.sched, k, it);
             ok = ptx::warp_all(ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ));
             if (!ok) break;
@@ -235,6 +280,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             }
         }
+        if (dynamic && lane == 0) p.work_counter[64 + blockIdx.x] = it;
         if (!ok) {
             // Leave no copy in flight: wait (briefly) for the loads issued last into each slot.
             if (q_issued) drain_wait(&bar->q_full, (q_issued - 1) & 1u);
@@ -293,7 +339,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const long long clk_begin = clock64();
             SAW_PROF_DECL;
             int it = 0;
-            for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+            for (; ok; ++it) {
+                const long long k = take_work(it, ok, false);
+                if (!ok || k < 0) break;
                 const WorkItem w = decode_work(p.sched, k, it);
                 const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
                 SAW_PROF(0);
@@ -382,7 +430,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         bool ok = true;
         int it = 0;
         SAW_PROF_DECL;
-        for (long long k = k_first; ok && k < p.sched.n_work; k += k_stride, ++it) {
+        for (; ok; ++it) {
+            const long long k = take_work(it, ok, true);
+            if (kSplit == 2 && dynamic) ok = ptx::bar_red_and(tile_bar, G::kTileThreads, ok);  // the tile's warps leave together
+            if (!ok || k < 0) break;
             const WorkItem w = decode_work(p.sched, k, it);
             const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
             if (hi_mine == 0) continue;

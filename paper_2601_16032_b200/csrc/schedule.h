@@ -25,6 +25,7 @@ struct SchedParams {
     int causal;       // 0 / 1
     int sawtooth;     // 0 = cyclic, 1 = sawtooth
     int head_fastest; // 0: k = (b*H + h)*n_q + t    1: k = (b*n_q + t)*H + h
+    int heavy_first;  // 1: digit t counts the Q blocks of a head from the last (most K/V tiles under the causal mask) to the first
     int n_q;          // work items per head = ceil(N / W)
     long long n_work; // B * H * n_q
 };
@@ -40,8 +41,10 @@ struct WorkItem {
 
 SAW_HD int ceil_div_i(int a, int b) { return (a + b - 1) / b; }
 
-SAW_HD SchedParams make_sched(int B, int H, int N, int q_tiles, int block_n, int causal, int sawtooth, int head_fastest) {
+SAW_HD SchedParams make_sched(int B, int H, int N, int q_tiles, int block_n, int causal, int sawtooth, int head_fastest,
+                              int heavy_first = 0) {
     SchedParams p;
+    p.heavy_first = heavy_first;
     p.B = B; p.H = H; p.N = N; p.q_tiles = q_tiles; p.block_n = block_n;
     p.causal = causal; p.sawtooth = sawtooth; p.head_fastest = head_fastest;
     p.n_q = ceil_div_i(N, q_tiles * kBlockM);
@@ -61,6 +64,7 @@ SAW_HD WorkItem decode_work(const SchedParams& p, long long k, int it) {
         w.q_item = (int)(r % p.n_q);
         w.bh = (int)(r / p.n_q) * p.H + h;
     }
+    if (p.heavy_first) w.q_item = p.n_q - 1 - w.q_item;
     w.row0 = w.q_item * p.q_tiles * kBlockM;
     w.backward = (p.sawtooth && (it & 1)) ? 1 : 0;
     const int n_kv = ceil_div_i(p.N, p.block_n);
