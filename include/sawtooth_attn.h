@@ -128,6 +128,29 @@ int attn_fwd_dynamic(const void* q, const void* k, const void* v, void* o,
                      void* scratch, size_t scratch_bytes);
 
 /*
+ * attn_fwd_dynamic for callers that cannot hand over scratch memory.  (The paper has no counterpart: this is a
+ * packaging of the dynamic schedule, not a step of the method.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- inside a region that is being recorded
+ * for replay, inside a framework's allocator callback, in a real-time loop with a no-allocation rule, or in a plug-in
+ * whose host application owns all device memory.  Such a caller has nowhere to get the counter buffer from, so here
+ * the buffer is a fixed array inside the library's own device image: ATTN_DYNAMIC_SCRATCH_HEADER + 4 *
+ * ATTN_NOALLOC_MAX_CTAS bytes (4352), present on every GPU the library is loaded on until the process exits.
+ * The call allocates and frees nothing; q, k, v, o are the caller's as everywhere else.
+ *
+ * Limits and rules.  A launch of more than ATTN_NOALLOC_MAX_CTAS persistent CTAs (grid of attn_query_plan) is
+ * refused with ATTN_ERR_INVALID_ARG before anything is enqueued.  The first call on each device looks up the
+ * array's address on that device (the device must be current); make that first call outside any stream capture.
+ * All calls on one device share the one array: it still holds the previous call's counters, every call clears them
+ * on `stream` before its kernel, and two calls that may run on the GPU at the same time (different streams) race
+ * on it -- serialise them, or use attn_fwd_dynamic with a buffer per stream.  Device indices up to 63.
+ */
+#define ATTN_NOALLOC_MAX_CTAS 1024
+int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* o,
+                             int B, int H, int N, int d, float scale, int causal, int scan_order,
+                             int dtype, void* stream, const attn_fwd_opts* opts);
+
+/*
  * Same computation for HOST buffers: copies q, k, v (host, ideally pinned) into the caller's device
  * staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host,
  * all enqueued on `stream`.  Each buffer holds B*H*N*d 16-bit elements.  Returns without waiting:

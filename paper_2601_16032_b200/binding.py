@@ -64,6 +64,8 @@ def load_library():
     lib.attn_fwd_ex.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts)]
     lib.attn_fwd_dynamic.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts), vp, ctypes.c_size_t]
     lib.attn_fwd_dynamic.restype = ci
+    lib.attn_fwd_dynamic_noalloc.argtypes = [vp, vp, vp, vp] + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts)]
+    lib.attn_fwd_dynamic_noalloc.restype = ci
     lib.attn_dynamic_scratch_bytes.argtypes = [ci]
     lib.attn_dynamic_scratch_bytes.restype = ctypes.c_size_t
     lib.attn_fwd_host.argtypes = [vp] * 8 + shape + [cf, ci, ci, ci, vp, ctypes.POINTER(Opts)]
@@ -121,6 +123,15 @@ def attn_fwd_dynamic(q: int, k: int, v: int, o: int, B: int, H: int, N: int, d: 
     """attn_fwd_ex with the dynamic tile schedule; scratch: device address of the caller's counter buffer."""
     _check(load_library().attn_fwd_dynamic(q, k, v, o, B, H, N, d, scale, int(causal), scan_order, dtype, stream,
                                            _opts_ptr(opts), scratch, scratch_bytes))
+
+
+def attn_fwd_dynamic_noalloc(q: int, k: int, v: int, o: int, B: int, H: int, N: int, d: int, scale: float, causal: int,
+                             scan_order: int, dtype: int, stream: int = 0, opts: Optional[Opts] = None) -> None:
+    """The dynamic schedule without a scratch argument, for callers that may not allocate device memory: the
+    counters live in a fixed array inside the library (at most 1024 CTAs; calls on one device share it, so calls
+    that could overlap on the GPU must be serialised; make the first call on a device outside stream capture)."""
+    _check(load_library().attn_fwd_dynamic_noalloc(q, k, v, o, B, H, N, d, scale, int(causal), scan_order, dtype, stream,
+                                                   _opts_ptr(opts)))
 
 
 def attn_fwd_host(q_host: int, k_host: int, v_host: int, o_host: int, q_dev: int, k_dev: int, v_dev: int, o_dev: int,

@@ -27,6 +27,12 @@ int fail(int status, const char* fmt, ...) {
 __device__ int g_status_word = 0;
 __device__ unsigned long long g_cycles = 0;
 
+// Scratch of attn_fwd_dynamic_noalloc: the claim counter block and one counter per CTA, resident in every GPU
+// that loads the library for as long as the process lives.
+static __device__ __align__(256) int g_noalloc_scratch[(ATTN_DYNAMIC_SCRATCH_HEADER / 4) + ATTN_NOALLOC_MAX_CTAS];
+constexpr int kMaxDevices = 64;
+int* g_noalloc_ptr[kMaxDevices] = {};  // device address of the array above, per device, once looked up
+
 constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
 
 struct Resolved {
@@ -267,6 +273,25 @@ int attn_fwd_dynamic(const void* q, const void* k, const void* v, void* o, int B
     const size_t ctas_max = (scratch_bytes - ATTN_DYNAMIC_SCRATCH_HEADER) / 4;
     return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, static_cast<int*>(scratch), scratch_bytes,
                       (int)(ctas_max < 2147483647u ? ctas_max : 2147483647u));
+}
+
+int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale,
+                             int causal, int scan_order, int dtype, void* stream, const attn_fwd_opts* opts) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
+    if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device index %d is beyond the %d this entry point keeps track of", dev, kMaxDevices);
+    if (!g_noalloc_ptr[dev]) {
+        // Set-up, once per device, with that device current.  In host code the array's name is only a handle for
+        // this lookup, not an address a kernel could use; the lookup gives the address inside the current device.
+        int* ptr = nullptr;
+        e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess || !ptr) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e)); }
+        g_noalloc_ptr[dev] = ptr;
+    }
+    // fwd_common turns a launch of more than ATTN_NOALLOC_MAX_CTAS CTAs away before anything is enqueued.
+    return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, g_noalloc_ptr[dev], sizeof(g_noalloc_scratch),
+                      ATTN_NOALLOC_MAX_CTAS);
 }
 
 static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
