@@ -286,6 +286,27 @@ def main():
                 acc[name].append(timed(lambda: step(orders[name]), 1))
         ab = {n: float(np.median(v)) for n, v in acc.items()}
 
+    # The dynamic tile schedule (work items claimed from a counter) beside the static one, same launches alternating.
+    dyn = None
+    if len(timed_orders) == 2:
+        plan0 = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt)
+        n_scratch = sa.attn_dynamic_scratch_bytes(plan0.grid)
+        scratch = torch.zeros(n_scratch // 4, dtype=torch.int32, device=dev)
+
+        def dyn_step(order):
+            sa.attn_fwd_dynamic(devb["q"].data_ptr(), devb["k"].data_ptr(), devb["v"].data_ptr(), devb["o"].data_ptr(),
+                                w.B, w.H, w.N, w.d, w.scale, int(w.causal), order, adt, sh, None, scratch.data_ptr(), n_scratch)
+
+        pairs = max(3, min(args.steps, 20))
+        acc = {"static": [], "dynamic": []}
+        for _ in range(3):
+            dyn_step(orders["sawtooth"])
+        for _ in range(pairs):
+            acc["static"].append(timed(lambda: step(orders["sawtooth"]), 1))
+            acc["dynamic"].append(timed(lambda: dyn_step(orders["sawtooth"]), 1))
+        sa.attn_device_status()
+        dyn = {n: float(np.median(v)) for n, v in acc.items()}
+
     # End to end: host buffers in, host buffer out, copies inside the timed region.
     e2e = None
     if not args.skip_e2e:
@@ -368,6 +389,10 @@ def main():
     if ab is not None:
         line["alternating_launches"] = {"cyclic_ms": ab["cyclic"], "sawtooth_ms": ab["sawtooth"],
                                         "sawtooth_over_cyclic": ab["cyclic"] / ab["sawtooth"]}
+    if dyn is not None:
+        line["dynamic_schedule"] = {"what": "attn_fwd_dynamic vs attn_fwd, sawtooth, single launches alternating",
+                                    "static_ms": dyn["static"], "dynamic_ms": dyn["dynamic"],
+                                    "dynamic_tflops": whole_job_tflops(flops, dyn["dynamic"], world)}
     if also:
         line["also"] = also
     if not args.skip_cpu_baseline:
