@@ -265,7 +265,7 @@ def main():
         return max_over_ranks(e0.elapsed_time(e1), dist, dev)
 
     orders = {"cyclic": sa.CYCLIC, "sawtooth": sa.SAWTOOTH}
-    timed_orders = ["cyclic", "sawtooth"] if args.scan_order == "both" else [args.scan_order]
+    timed_orders = ["sawtooth", "cyclic"] if args.scan_order == "both" else [args.scan_order]  # the headline order first
     headline = "sawtooth" if "sawtooth" in timed_orders else "cyclic"
     results = {}
     with ClockSampler(local) as clocks:
