@@ -191,6 +191,7 @@ def main():
     ap.add_argument("--scan-order", default="both", choices=["both", "cyclic", "sawtooth"],
                     help="orders to time; `value` is the sawtooth order unless only cyclic is timed")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--max-ctas", type=int, default=0, help="cap on the persistent grid (the paper's 'active SMs'); 0 = all SMs")
     ap.add_argument("--also", default="c2,c4,c5",
                     help="further workloads timed briefly in both orders (single GPU only; '' for none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -239,10 +240,15 @@ def main():
     stream = torch.cuda.Stream(device=dev)
     sh = stream.cuda_stream
 
+    run_opts = None
+    if args.max_ctas > 0:
+        run_opts = sa.Opts()
+        run_opts.max_ctas = args.max_ctas
+
     def make_step(bufs, wk, a_dt):
         def step(order):
-            sa.attn_fwd(bufs["q"].data_ptr(), bufs["k"].data_ptr(), bufs["v"].data_ptr(), bufs["o"].data_ptr(),
-                        wk.B, wk.H, wk.N, wk.d, wk.scale, int(wk.causal), order, a_dt, sh)
+            sa.attn_fwd_ex(bufs["q"].data_ptr(), bufs["k"].data_ptr(), bufs["v"].data_ptr(), bufs["o"].data_ptr(),
+                           wk.B, wk.H, wk.N, wk.d, wk.scale, int(wk.causal), order, a_dt, sh, run_opts)
         return step
 
     step = make_step(devb, w, adt)
@@ -364,7 +370,7 @@ def main():
     timed_region_s = ms_head * args.steps / 1e3
     peak_kind = "sustained" if timed_region_s >= 0.5 else "burst"
     peak = peaks[peak_kind]
-    plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt)
+    plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt, run_opts)
     line = {
         "metric": METRIC, "value": whole_job_tflops(flops, ms_head, world), "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_head, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

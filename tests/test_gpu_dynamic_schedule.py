@@ -42,6 +42,19 @@ def test_dynamic_schedule_parity_and_coverage(causal, d, dtype, max_ctas):
         assert scratch[0] == plan.n_work + plan.grid                      # plus one failed claim per CTA
 
 
+@pytest.mark.parametrize("block_n,q_tiles", [(64, 2), (128, 1), (64, 1)])
+@pytest.mark.parametrize("N", [1, 129, 1000])
+def test_dynamic_schedule_other_tile_shapes_and_sizes(block_n, q_tiles, N):
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("dyn-shapes", 1, 5, N, 128, wl.BF16, True, 7450 + N)
+    qkv = upload(w)
+    opts = sa.Opts()
+    opts.block_n, opts.q_tiles, opts.max_ctas = block_n, q_tiles, 2
+    o, scratch, plan = run_dynamic(w, qkv, sa.SAWTOOTH, opts)
+    assert_parity(w, o)
+    assert scratch[64:64 + plan.grid].sum() == plan.n_work
+
+
 def test_dynamic_cyclic_equals_static_bitwise():
     import torch
     import paper_2601_16032_b200 as sa

@@ -65,7 +65,11 @@ CONFIGS = {
 STUDY_CASES = {
     "c3-small": Workload("c3-small", 2, 16, 8192, 128, BF16, False, 2003),
     "c4-small": Workload("c4-small", 1, 8, 32768, 128, BF16, True, 2004, k_scale=0.5),
+    "long-64k": Workload("long-64k", 1, 1, 65536, 128, BF16, False, 2010),
+    "long-128k": Workload("long-128k", 1, 1, 131072, 128, BF16, False, 2011),
+    "long-192k": Workload("long-192k", 1, 1, 196608, 128, BF16, False, 2012),
     "long-256k": Workload("long-256k", 1, 1, 262144, 128, BF16, False, 2006),
+    "long-384k": Workload("long-384k", 1, 1, 393216, 128, BF16, False, 2013),
     "long-512k": Workload("long-512k", 1, 1, 524288, 128, BF16, False, 2007),
     "long-128k-b8": Workload("long-128k-b8", 8, 1, 131072, 64, F16, False, 2008),
 }
