@@ -102,6 +102,25 @@ def test_invariants_on_gpu():
     assert (o - v[:, :, 123:124]).abs().max() < 2e-2
 
 
+def test_cycle_counter_reports_a_plausible_clock():
+    """attn_last_kernel_cycles / elapsed time is an SM clock between 0.5 and 2.2 GHz for a launch that fills the GPU."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    q = torch.randn(2, 16, 4096, 128, device="cuda:0").to(torch.bfloat16)
+    o = torch.empty_like(q)
+    st = torch.cuda.current_stream().cuda_stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        if i == 2:
+            e0.record()
+        sa.attn_fwd(q.data_ptr(), q.data_ptr(), q.data_ptr(), o.data_ptr(), 2, 16, 4096, 128, 0.088, 0, sa.SAWTOOTH, sa.BF16, st)
+    e1.record()
+    cycles = sa.attn_last_kernel_cycles()
+    sa.attn_device_status()
+    mhz = cycles / (e0.elapsed_time(e1) * 1e3)
+    assert 500 < mhz < 2200, (cycles, e0.elapsed_time(e1))
+
+
 def test_bad_arguments_are_rejected_before_launch():
     import torch
     import paper_2601_16032_b200 as sa
