@@ -142,33 +142,33 @@ int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, i
 }
 
 template <int kD, int kBlockN, int kQTiles, int kBf16>
-int launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const KernelParams& kp, int grid,
+int launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const KernelParams& kp, int grid,
            size_t smem, cudaStream_t stream) {
     auto kern = attn_fwd_kernel<kD, kBlockN, kQTiles, kBf16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); }
-    kern<<<grid, Geometry<kD, kBlockN, kQTiles>::kThreads, smem, stream>>>(tq, tk, tv, kp);
+    kern<<<grid, Geometry<kD, kBlockN, kQTiles>::kThreads, smem, stream>>>(tq, tk, tv, to, kp);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
     return ATTN_OK;
 }
 
 template <int kD, int kBlockN, int kQTiles>
-int launch_dtype(int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const KernelParams& kp,
+int launch_dtype(int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const KernelParams& kp,
                  int grid, size_t smem, cudaStream_t stream) {
-    return dtype == ATTN_BF16 ? launch<kD, kBlockN, kQTiles, 1>(tq, tk, tv, kp, grid, smem, stream)
-                              : launch<kD, kBlockN, kQTiles, 0>(tq, tk, tv, kp, grid, smem, stream);
+    return dtype == ATTN_BF16 ? launch<kD, kBlockN, kQTiles, 1>(tq, tk, tv, to, kp, grid, smem, stream)
+                              : launch<kD, kBlockN, kQTiles, 0>(tq, tk, tv, to, kp, grid, smem, stream);
 }
 
 template <int kD>
 int launch_tiles(int block_n, int q_tiles, int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                 const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
+                 const CUtensorMap& to, const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
     if (block_n == 128) {
-        return q_tiles == 2 ? launch_dtype<kD, 128, 2>(dtype, tq, tk, tv, kp, grid, smem, stream)
-                            : launch_dtype<kD, 128, 1>(dtype, tq, tk, tv, kp, grid, smem, stream);
+        return q_tiles == 2 ? launch_dtype<kD, 128, 2>(dtype, tq, tk, tv, to, kp, grid, smem, stream)
+                            : launch_dtype<kD, 128, 1>(dtype, tq, tk, tv, to, kp, grid, smem, stream);
     }
-    return q_tiles == 2 ? launch_dtype<kD, 64, 2>(dtype, tq, tk, tv, kp, grid, smem, stream)
-                        : launch_dtype<kD, 64, 1>(dtype, tq, tk, tv, kp, grid, smem, stream);
+    return q_tiles == 2 ? launch_dtype<kD, 64, 2>(dtype, tq, tk, tv, to, kp, grid, smem, stream)
+                        : launch_dtype<kD, 64, 1>(dtype, tq, tk, tv, to, kp, grid, smem, stream);
 }
 
 }  // namespace
@@ -331,6 +331,10 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
     if ((rc = make_map(&tq, q, B * H, N, d, kBlockM, dtype))) return rc;
     if ((rc = make_map(&tk, k, B * H, N, d, r.block_n, dtype))) return rc;
     if ((rc = make_map(&tv, v, B * H, N, d, r.block_n, dtype))) return rc;
+    // O is written through shared memory in boxes of 64 columns x as many rows as one warp's share of a ring slot holds.
+    CUtensorMap to;
+    const int stage_rows = (r.block_n * d * 2 / 2 / 4) / 128 < 32 ? (r.block_n * d * 2 / 2 / 4) / 128 : 32;
+    if ((rc = make_map(&to, o, B * H, N, d, stage_rows, dtype))) return rc;
 
     const int grid = grid_for(kp.sched.n_work, sm_count, r);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -343,8 +347,8 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
         cudaError_t e = cudaMemsetAsync(work_counter, 0, (size_t)ATTN_DYNAMIC_SCRATCH_HEADER + 4u * (size_t)grid, st);
         if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "clearing the scratch: %s", cudaGetErrorString(e)); }
     }
-    return d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st)
-                    : launch_tiles<64>(r.block_n, r.q_tiles, dtype, tq, tk, tv, kp, grid, r.smem, st);
+    return d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, tq, tk, tv, to, kp, grid, r.smem, st)
+                    : launch_tiles<64>(r.block_n, r.q_tiles, dtype, tq, tk, tv, to, kp, grid, r.smem, st);
 }
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,

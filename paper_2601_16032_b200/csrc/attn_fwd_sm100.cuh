@@ -61,7 +61,8 @@ constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the
 // Codes written to the status word: which wait gave up.
 enum WaitSite {
     kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
-    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8, kSiteWorkFull = 9, kSiteWorkEmpty = 10
+    kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8, kSiteWorkFull = 9, kSiteWorkEmpty = 10,
+    kSiteStageSlot = 11, kSiteStageDone = 12
 };
 
 struct __align__(8) Barriers {
@@ -69,6 +70,7 @@ struct __align__(8) Barriers {
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
     uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
     uint64_t drain[2];
+    uint64_t stage_done[2];                 // staged epilogue: the four warps of Q tile q have read their staging buffers out
     uint64_t work_full[2], work_empty[2];  // dynamic schedule: two-slot mailbox of claimed work indices
     long long work_k[2];
     uint32_t tmem_base;
@@ -88,6 +90,13 @@ struct Geometry {
     static constexpr int kColsO = kD / kSplit;              // O columns a softmax thread owns
     // P reaches the MMA warp in two parts: a thread announces its first kEarlyGroups groups of 16
     // probabilities (one K step of the P.V product each) while it still computes the rest.
+    // Epilogue through shared memory: after the last V tile of a work item the ring holds one more slot that
+    // nothing is loaded into; the softmax warps of Q tile q stage their 16-bit O rows in half q of it, kStageRows rows
+    // of one 64-column block per warp at a time, and write them out with TMA stores (full 128-byte lines, rows
+    // beyond N dropped by the copy engine).  Only with one thread per row.
+    static constexpr bool kStagedEpilogue = (kSplit == 1);
+    static constexpr int kStageBytesPerWarp = kKVTileBytes / 2 / 4;
+    static constexpr int kStageRows = kStageBytesPerWarp / 128 < 32 ? kStageBytesPerWarp / 128 : 32;
     static constexpr int kGroups = kColsS / 16;
     static constexpr int kEarlyGroups = kGroups >= 4 ? (kGroups * 3) / 4 : kGroups / 2;
     static constexpr int kSoftmaxWarps = kQTiles * kSplit * 4;
@@ -114,6 +123,11 @@ struct Ring {
     __device__ __forceinline__ void advance(int stages) {
         if (++slot == stages) { slot = 0; phase ^= 1u; }
     }
+    __device__ __forceinline__ void advance_by(int n, int stages) {
+        const int t = slot + n;
+        slot = t % stages;
+        phase ^= (uint32_t)(t / stages) & 1u;
+    }
 };
 
 // Short wait that ignores the abort flag: used on the way out, for copies and MMAs still in flight.
@@ -127,7 +141,7 @@ __device__ __forceinline__ void drain_wait(uint64_t* bar, uint32_t parity) {
 template <int kD, int kBlockN, int kQTiles, int kBf16>
 __global__ void __launch_bounds__(Geometry<kD, kBlockN, kQTiles>::kThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const KernelParams p)
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const KernelParams p)
 {
     using G = Geometry<kD, kBlockN, kQTiles>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -164,6 +178,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ptx::mbar_init(&bar->work_full[i], 1);
             ptx::mbar_init(&bar->work_empty[i], kQTiles + G::kSoftmaxWarps);
         }
+        ptx::mbar_init(&bar->stage_done[0], 4);
+        ptx::mbar_init(&bar->stage_done[1], 4);
         ptx::mbar_init(&bar->drain[0], 1);
         ptx::mbar_init(&bar->drain[1], 1);
         bar->abort_flag = 0;
@@ -173,6 +189,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ptx::prefetch_tmap(&tm_q);
         ptx::prefetch_tmap(&tm_k);
         ptx::prefetch_tmap(&tm_v);
+        ptx::prefetch_tmap(&tm_o);
     }
     if (warp == kMmaWarp) {
         ptx::tmem_alloc(&bar->tmem_base, G::kTmemCols);
@@ -278,6 +295,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ring.advance(stages);
                     ++kv_issued;
                 }
+            }
+            if (ok && G::kStagedEpilogue) {
+                // The item's staging slot: wait until its last contents are consumed, then hand it to the softmax warps
+                // through the slot's own full barrier (no bytes are expected).
+                ok = ptx::warp_all(ptx::mbar_wait(&bar->kv_empty[ring.slot], ring.phase ^ 1u, abort_flag, kSiteProducerKV));
+                if (!ok) break;
+                if (ptx::elect_one()) ptx::mbar_arrive(&bar->kv_full[ring.slot]);
+                __syncwarp();
+                ring.advance(stages);
+                ++kv_issued;
             }
         }
         if (dynamic && lane == 0) p.work_counter[64 + blockIdx.x] = it;
@@ -401,6 +428,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (!ok) break;
                 if (hi_mine > 0) ptx::mma_commit(&bar->o_full[q]);
+                if (G::kStagedEpilogue) {
+                    // The staging slot is released by the tile's softmax warps, or here if the tile lies beyond N.
+                    if (hi_mine == 0) ptx::mbar_arrive(&bar->kv_empty[ring.slot]);
+                    ring.advance(stages);
+                }
             }
             // Nothing of this thread's MMAs may be in flight when TMEM is released.
             ptx::mma_commit(&bar->drain[q]);
@@ -429,6 +461,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t s_phase = 0, o_phase = 0;
         bool ok = true;
         int it = 0;
+        Ring ring;                 // position of the next work item's first K tile in the K/V ring
+        uint32_t stage_phase = 0;
         SAW_PROF_DECL;
         for (; ok; ++it) {
             const long long k = take_work(it, ok, true);
@@ -436,6 +470,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok || k < 0) break;
             const WorkItem w = decode_work(p.sched, k, it);
             const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
+            ring.advance_by(2 * w.hi, stages);   // now at the item's staging slot
+            const Ring stage = ring;
+            ring.advance(stages);
             if (hi_mine == 0) continue;
             const int tile_row0 = w.row0 + q * kBlockM;
             const int row = tile_row0 + r_in_tile;
@@ -584,6 +621,53 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (!ok) break;
             }
             const float inv_l = 1.f / l;
+            if (G::kStagedEpilogue) {
+                ok = ptx::warp_all(ptx::mbar_wait(&bar->kv_full[stage.slot], stage.phase, abort_flag, kSiteStageSlot));
+                if (!ok) break;
+                uint8_t* buf = kv_smem + (size_t)stage.slot * G::kKVTileBytes + (size_t)q * (G::kKVTileBytes / 2) +
+                               (size_t)(warp & 3) * G::kStageBytesPerWarp;
+                const int my_pass = lane / G::kStageRows, my_row = lane % G::kStageRows;
+#pragma unroll
+                for (int c64 = 0; c64 < kD / 64; ++c64) {
+                    uint32_t pk[32];   // this row's 64 columns of the block, 16-bit pairs
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        uint32_t ov[32];
+                        ptx::tmem_ld32(t_o + c64 * 64 + hf * 32, ov);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2)
+                            pk[hf * 16 + i / 2] = ptx::pack2<kBf16>(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l);
+                    }
+#pragma unroll 1
+                    for (int ps = 0; ps < 32 / G::kStageRows; ++ps) {
+                        if (my_pass == ps) {
+                            // 128-byte rows, eight to a 1024-byte swizzle atom: 16-byte piece i of row r sits at piece i ^ (r & 7)
+                            uint4* dst_row = reinterpret_cast<uint4*>(buf + my_row * 128);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                dst_row[i ^ (my_row & 7)] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        const int y0 = tile_row0 + (warp & 3) * 32 + ps * G::kStageRows;
+                        if (y0 < N && ptx::elect_one()) {   // rows of the box beyond N are dropped by the copy
+                            ptx::tma_store_3d(&tm_o, buf, c64 * 64, y0, w.bh);
+                            ptx::bulk_commit_group();
+                            ptx::bulk_wait_group_read0();   // the buffer may be written again
+                        }
+                        __syncwarp();
+                    }
+                }
+                // The slot goes back to the producer once the four warps of the tile have read their buffers out.
+                if (lane == 0) ptx::mbar_arrive(&bar->stage_done[q]);
+                if ((warp & 3) == 0) {
+                    ok = ptx::warp_all(ptx::mbar_wait(&bar->stage_done[q], stage_phase, abort_flag, kSiteStageDone));
+                    if (ok && lane == 0) ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
+                }
+                stage_phase ^= 1u;
+                if (!ok) break;
+            } else {
             uint4* o_row = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.o) + ((size_t)w.bh * N + row) * (size_t)(kD * 2) +
                                                     (size_t)half * (kColsO * 2));
 #pragma unroll
@@ -601,11 +685,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         o_row[c * 4 + v4] = make_uint4(pk[4 * v4], pk[4 * v4 + 1], pk[4 * v4 + 2], pk[4 * v4 + 3]);
                 }
             }
+            }
             ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
             // The other thread of the row has read this thread's partial sum before the buffer holds a maximum again.
             if (kSplit == 2) ptx::bar_sync(tile_bar, G::kTileThreads);
             SAW_PROF(8);
         }
+        if (G::kStagedEpilogue) ptx::bulk_wait_group0();   // this thread's TMA stores have landed before the CTA ends
         SAW_PROF_WRITE(12, q == 0 && half == 0 && r_in_tile == 0);
     }
 
