@@ -37,9 +37,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes one launch of the bench workload moves (dram__bytes_read.sum + dram__bytes_write.sum of
 # an ncu capture of the same kernel; see the summary under profiles/).  None until captured.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    # c3-small (half of c3's heads, same kernel): 201,864,704 B read + 43,682,048 B written, scaled by 2 heads-wise
-    "c3": 2 * (201864704 + 43682048),
-    "c3-small": 201864704 + 43682048,
+    # c3-small (half of c3's heads, same kernel): 202,101,760 B read + 47,526,144 B written, scaled by 2 heads-wise
+    "c3": 2 * (202101760 + 47526144),
+    "c3-small": 202101760 + 47526144,
 }
 
 
