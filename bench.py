@@ -347,7 +347,8 @@ def main():
             if wk.k_scale != 1.0:
                 bufs["k"] *= wk.k_scale
             bufs["o"] = torch.empty_like(bufs["q"])
-            st = make_step(bufs, wk, sa.BF16 if wk.dtype == wl.BF16 else sa.F16)
+            a_dt = sa.BF16 if wk.dtype == wl.BF16 else sa.F16
+            st = make_step(bufs, wk, a_dt)
             n_steps = max(3, min(args.steps, int(200.0 / (wk.flops / 1e12))))  # about 0.2 s per order
             entry = {"workload": config_of(wk)["workload"], "steps": n_steps}
             for oname in ("cyclic", "sawtooth"):
@@ -355,6 +356,17 @@ def main():
                     st(orders[oname])
                 ms = timed(lambda: st(orders[oname]), n_steps) / n_steps
                 entry[oname] = {"value": wk.flops / ms / 1e9, "unit": UNIT, "ms_per_step": ms}
+            n_scr = sa.attn_dynamic_scratch_bytes(sa.attn_query_plan(wk.B, wk.H, wk.N, wk.d, int(wk.causal), a_dt).grid)
+            scr = torch.zeros(n_scr // 4, dtype=torch.int32, device=dev)
+
+            def dyn_also(order, bufs=bufs, wk=wk, a_dt=a_dt, scr=scr, n_scr=n_scr):
+                sa.attn_fwd_dynamic(bufs["q"].data_ptr(), bufs["k"].data_ptr(), bufs["v"].data_ptr(), bufs["o"].data_ptr(),
+                                    wk.B, wk.H, wk.N, wk.d, wk.scale, int(wk.causal), order, a_dt, sh, None, scr.data_ptr(), n_scr)
+
+            for _ in range(3):
+                dyn_also(orders["sawtooth"])
+            ms = timed(lambda: dyn_also(orders["sawtooth"]), n_steps) / n_steps
+            entry["sawtooth_dynamic_schedule"] = {"value": wk.flops / ms / 1e9, "unit": UNIT, "ms_per_step": ms}
             sa.attn_device_status()
             also[name] = entry
             del bufs

@@ -60,3 +60,42 @@ def test_c4_causal_two_heads_plus_sampled_rows():
 
 def test_c5_causal_sampled_rows_every_head():
     check_config("c5", [("default", None)])
+
+
+def test_long_single_head_beyond_l2_sampled_rows():
+    """One head of 262,144 keys (K+V = 128 MiB, more than the L2): 256 seeded rows plus the tile-edge rows, both scan
+    orders and the dynamic schedule, against the oracle."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.STUDY_CASES["long-256k"]
+    plan = {(0, 0): wl.sampled_rows(w, 0, 0, 256)}
+    want = oracle_rows(w, plan)
+    qkv = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        o = run_cuda(w, qkv, order)
+        max_abs, mean_abs, n_rows = compare_rows(w, o, plan, want)
+        assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, (order, max_abs, mean_abs, n_rows)
+    q, k, v = qkv
+    n_bytes = sa.attn_dynamic_scratch_bytes(sa.attn_query_plan(w.B, w.H, w.N, w.d, 0, sa.BF16).grid)
+    scratch = torch.zeros(n_bytes // 4, dtype=torch.int32, device=q.device)
+    o = torch.full_like(q, float("nan"))
+    sa.attn_fwd_dynamic(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, 0, sa.SAWTOOTH, sa.BF16,
+                        torch.cuda.current_stream().cuda_stream, None, scratch.data_ptr(), n_bytes)
+    sa.attn_device_status()
+    max_abs, mean_abs, n_rows = compare_rows(w, o, plan, want)
+    assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, ("dynamic", max_abs, mean_abs, n_rows)
+
+
+def test_many_small_heads():
+    """1,500 heads of 300 keys: many more (batch, head) pairs than SMs, ragged length, both tile shapes."""
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("many-heads", 25, 60, 300, 64, wl.F16, True, 7900)
+    plan = {(b, h): None for (b, h) in [(0, 0), (7, 31), (24, 59)]}
+    want = oracle_rows(w, plan)
+    qkv = upload(w)
+    for block_n in (128, 64):
+        opts = sa.Opts()
+        opts.block_n = block_n
+        o = run_cuda(w, qkv, sa.SAWTOOTH, opts)
+        max_abs, mean_abs, _ = compare_rows(w, o, plan, want)
+        assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, (block_n, max_abs, mean_abs)
