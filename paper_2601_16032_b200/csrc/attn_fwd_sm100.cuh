@@ -1,22 +1,24 @@
 // FlashAttention forward kernel for sm_100a: persistent CTAs, TMA-fed K/V ring, tcgen05 MMAs with
-// S, P and O in tensor memory, one softmax thread per query row.
+// S, P and O in tensor memory, one softmax thread per query row, O written by TMA stores.
 //
 // One CTA handles work items of kQTiles x 128 query rows (Algorithm 1's resident Q tile).  Warp roles:
 //   the softmax warps      one warpgroup per Q tile, thread r owning row r (TMEM lane r), or, built with
 //                          SAW_THREADS_PER_ROW=2, two warpgroups per tile whose threads split a row's
 //                          columns and exchange their row maxima through shared memory.  A thread reads
 //                          its part of S from TMEM, keeps the running max and a (partial) sum, writes P
-//                          back to TMEM as 16-bit pairs, rescales its part of O when the max moved, and
-//                          at the end of the item normalises and stores its part of the O row.
+//                          back to TMEM as 16-bit pairs in two parts, rescales its part of O when the max
+//                          moved, and at the end of the item normalises its part of the O row and stages
+//                          it in shared memory, from where one lane per warp issues a TMA store.
 //   the next warp          producer: one elected lane issues the TMA loads (Q tiles, then K_j, V_j in
-//                          the scan order of the item) into a ring of shared-memory slots.
+//                          the scan order of the item, then one empty slot: the item's O staging buffer)
+//                          into a ring of shared-memory slots.
 //   the next kQTiles warps MMA, one warp per Q tile q: one elected lane issues S_q = Q_q K_j^T and
 //                          O_q += P_q V_j and commits them to mbarriers; the first of them also owns
 //                          the TMEM allocation.
 //   the remaining warp(s)  idle; they complete the warpgroup whose registers go to the softmax threads.
 // With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
-// Four softmax warps per scheduler (two threads per row) keep the MUFU busy: one warp alone can start
-// an exponential only every other MUFU slot.
+// Work items come from Algorithm 2's grid-stride walk or, with a counter in global memory, are claimed
+// dynamically; Algorithm 4's scan direction follows the CTA's own item count either way.
 #pragma once
 #include "ptx.cuh"
 #include "schedule.h"
@@ -88,8 +90,6 @@ struct Geometry {
     static constexpr int kSplit = SAW_THREADS_PER_ROW;      // threads per query row (1 or 2)
     static constexpr int kColsS = kBlockN / kSplit;         // S columns a softmax thread owns
     static constexpr int kColsO = kD / kSplit;              // O columns a softmax thread owns
-    // P reaches the MMA warp in two parts: a thread announces its first kEarlyGroups groups of 16
-    // probabilities (one K step of the P.V product each) while it still computes the rest.
     // Epilogue through shared memory: after the last V tile of a work item the ring holds one more slot that
     // nothing is loaded into; the softmax warps of Q tile q stage their 16-bit O rows in half q of it, kStageRows rows
     // of one 64-column block per warp at a time, and write them out with TMA stores (full 128-byte lines, rows
@@ -97,11 +97,13 @@ struct Geometry {
     static constexpr bool kStagedEpilogue = (kSplit == 1);
     static constexpr int kStageBytesPerWarp = kKVTileBytes / 2 / 4;
     static constexpr int kStageRows = kStageBytesPerWarp / 128 < 32 ? kStageBytesPerWarp / 128 : 32;
+    // P reaches the MMA warp in two parts: a thread announces its first kEarlyGroups groups of 16
+    // probabilities (one K step of the P.V product each) while it still computes the rest.
     static constexpr int kGroups = kColsS / 16;
     static constexpr int kEarlyGroups = kGroups >= 4 ? (kGroups * 3) / 4 : kGroups / 2;
     static constexpr int kSoftmaxWarps = kQTiles * kSplit * 4;
     static constexpr int kTileThreads = 128 * kSplit;       // threads that share one Q tile (one named barrier)
-    static constexpr int kThreads = kSoftmaxWarps * 32 + 128;  // plus one warpgroup: producer, MMA, two idle warps
+    static constexpr int kThreads = kSoftmaxWarps * 32 + 128;  // plus one warpgroup: producer, MMA warps, idle warp(s)
     // Registers: the launch gives every thread 65536 / kThreads rounded down to a multiple of 8.  With
     // two Q tiles that is 96 (640 threads, two per row) or 168 (384 threads, one per row): the last
     // warpgroup hands registers back and the softmax warpgroups take them
@@ -239,7 +241,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     };
 
     if (warp >= G::kSoftmaxWarps) {
-    // The last warpgroup (producer, MMA and two idle warps) hands registers back in one instruction.
+    // The last warpgroup (producer, MMA and idle warps) hands registers back in one instruction.  (Its three
+    // roles below keep the indentation of the outer level.)
     if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
