@@ -611,9 +611,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             if (!ok) break;
             // ---- epilogue: O_q / l -> 16 bit -> global
+            SAW_PROF(0);
             const bool got_o = ptx::mbar_wait(&bar->o_full[q], o_phase, abort_flag, kSiteSoftmaxO);
             o_phase ^= 1u;
             ptx::tc_fence_after();
+            SAW_PROF(9);
             if (kSplit == 2) {
                 *xchg_mine = l;
                 ok = ptx::bar_red_and(tile_bar, G::kTileThreads, got_o);
@@ -627,6 +629,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (G::kStagedEpilogue) {
                 ok = ptx::warp_all(ptx::mbar_wait(&bar->kv_full[stage.slot], stage.phase, abort_flag, kSiteStageSlot));
                 if (!ok) break;
+                SAW_PROF(10);
                 uint8_t* buf = kv_smem + (size_t)stage.slot * G::kKVTileBytes + (size_t)q * (G::kKVTileBytes / 2) +
                                (size_t)(warp & 3) * G::kStageBytesPerWarp;
                 const int my_pass = lane / G::kStageRows, my_row = lane % G::kStageRows;
@@ -662,6 +665,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         __syncwarp();
                     }
                 }
+                SAW_PROF(11);
                 // The slot goes back to the producer once the four warps of the tile have read their buffers out.
                 if (lane == 0) ptx::mbar_arrive(&bar->stage_done[q]);
                 if ((warp & 3) == 0) {
