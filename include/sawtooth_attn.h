@@ -63,7 +63,8 @@ typedef struct {
     int digit_order;  /* attn_digit_order: how the linear work index maps to (batch, head, Q block) */
     int launch_mode;  /* 0: persistent grid (Algorithm 2); 1: one CTA per work item (Algorithm 3) */
     int l2_policy;    /* 0: no hint; 1: K/V loads carry an evict_last hint, Q loads evict_first */
-    int reserved[9];
+    int host_chunks;  /* attn_fwd_host only: pieces the heads are cut into so that copies and kernels overlap (1..16; 0 = automatic) */
+    int reserved[8];
 } attn_fwd_opts;
 
 /* What a call with these arguments will launch; lets a caller predict L2 traffic. */
@@ -151,10 +152,14 @@ int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* 
                              int dtype, void* stream, const attn_fwd_opts* opts);
 
 /*
- * Same computation for HOST buffers: copies q, k, v (host, ideally pinned) into the caller's device
- * staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host,
- * all enqueued on `stream`.  Each buffer holds B*H*N*d 16-bit elements.  Returns without waiting:
- * o_host is valid once the stream has been synchronised.
+ * Same computation for HOST buffers: copies q, k, v (host, pinned if the copies are to overlap anything) into the
+ * caller's device staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host.
+ * Each buffer holds B*H*N*d 16-bit elements.  The heads are independent, so the work is cut into opts->host_chunks
+ * groups of heads (automatic: up to 8 once a tensor exceeds 32 MiB) that run as a pipeline on three streams the
+ * library keeps per device: upload of group i+1, kernel of group i and download of group i-1 proceed together.  The
+ * pipeline starts after everything already enqueued on `stream` and `stream` waits for its end, so to the caller it
+ * behaves like work enqueued on `stream`.  Returns without waiting: o_host is valid once `stream` has been
+ * synchronised.  The first pipelined call on a device creates the streams and events (no device memory).
  */
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
                   void* q_dev, void* k_dev, void* v_dev, void* o_dev,

@@ -25,7 +25,7 @@ class Opts(ctypes.Structure):
     _fields_ = [
         ("max_ctas", ctypes.c_int), ("kv_stages", ctypes.c_int), ("block_n", ctypes.c_int),
         ("q_tiles", ctypes.c_int), ("digit_order", ctypes.c_int), ("launch_mode", ctypes.c_int),
-        ("l2_policy", ctypes.c_int), ("reserved", ctypes.c_int * 9),
+        ("l2_policy", ctypes.c_int), ("host_chunks", ctypes.c_int), ("reserved", ctypes.c_int * 8),
     ]
 
 

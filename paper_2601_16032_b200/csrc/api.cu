@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/sawtooth_attn.h"
 #include "attn_fwd_sm100.cuh"
@@ -33,6 +34,7 @@ static __device__ __align__(256) int g_noalloc_scratch[(ATTN_DYNAMIC_SCRATCH_HEA
 constexpr int kMaxDevices = 64;
 int* g_noalloc_ptr[kMaxDevices] = {};  // device address of the array above, per device, once looked up
 
+constexpr int kMaxHostChunks = 16;
 constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
 
 struct Resolved {
@@ -67,6 +69,7 @@ int resolve_opts(const attn_fwd_opts* o, int d, int smem_limit, Resolved* r) {
     if (z.launch_mode != 0 && z.launch_mode != 1) return fail(ATTN_ERR_INVALID_ARG, "launch_mode must be 0 or 1");
     if (z.l2_policy != 0 && z.l2_policy != 1) return fail(ATTN_ERR_INVALID_ARG, "l2_policy must be 0 or 1");
     if (z.max_ctas < 0 || z.kv_stages < 0) return fail(ATTN_ERR_INVALID_ARG, "max_ctas and kv_stages must be >= 0");
+    if (z.host_chunks < 0 || z.host_chunks > kMaxHostChunks) return fail(ATTN_ERR_INVALID_ARG, "host_chunks must be in [0, %d]", kMaxHostChunks);
     r->head_fastest = z.digit_order == ATTN_HEAD_FASTEST;
     r->launch_mode = z.launch_mode;
     r->l2_policy = z.l2_policy;
@@ -356,6 +359,40 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H,
     return attn_fwd_ex(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, nullptr);
 }
 
+namespace {
+// Streams and events of the attn_fwd_host pipeline, one set per device, created on first use.
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t up = nullptr, run = nullptr, down = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, uploaded[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {};
+};
+HostPipe g_host_pipe[kMaxDevices];
+std::mutex g_host_pipe_mutex;
+
+int host_pipe_for_current_device(HostPipe** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
+    if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device index %d is beyond the %d the host pipeline keeps track of", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
+    HostPipe& hp = g_host_pipe[dev];
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.run, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kMaxHostChunks; ++i)
+            ok = cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "creating the streams and events of the host pipeline failed"); }
+        hp.ready = true;
+    }
+    *out = &hp;
+    return ATTN_OK;
+}
+}  // namespace
+
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, void* q_dev, void* k_dev,
                   void* v_dev, void* o_dev, int B, int H, int N, int d, float scale, int causal, int scan_order, int dtype,
                   void* stream, const attn_fwd_opts* opts) {
@@ -366,18 +403,57 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     const size_t bytes = (size_t)B * H * N * d * 2;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(v_dev, v_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(ATTN_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
+    const long long heads = (long long)B * H;
+    int chunks = opts ? opts->host_chunks : 0;
+    if (chunks < 0 || chunks > kMaxHostChunks) return fail(ATTN_ERR_INVALID_ARG, "host_chunks must be in [0, %d]", kMaxHostChunks);
+    if (chunks == 0) chunks = bytes > ((size_t)32 << 20) ? 8 : 1;
+    if (chunks > heads) chunks = (int)heads;
+    if (chunks <= 1) {
+        if ((e = cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(v_dev, v_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ATTN_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
+        }
+        rc = attn_fwd_ex(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, stream, opts);
+        if (rc) return rc;
+        if ((e = cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(ATTN_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
+        }
+        return ATTN_OK;
     }
-    rc = attn_fwd_ex(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, stream, opts);
-    if (rc) return rc;
-    if ((e = cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(ATTN_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
+    // Pipeline over groups of heads: upload, kernel and download of successive groups overlap on three streams.
+    HostPipe* hp = nullptr;
+    if ((rc = host_pipe_for_current_device(&hp))) return rc;
+    const size_t head_bytes = (size_t)N * d * 2;
+    auto fail_cuda = [&](const char* what) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e)); };
+    if ((e = cudaEventRecord(hp->start, st)) != cudaSuccess) return fail_cuda("cudaEventRecord");
+    if ((e = cudaStreamWaitEvent(hp->up, hp->start, 0)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->run, hp->start, 0)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->down, hp->start, 0)) != cudaSuccess)
+        return fail_cuda("cudaStreamWaitEvent");
+    long long h0 = 0;
+    for (int c = 0; c < chunks; ++c) {
+        const long long n_heads = heads / chunks + (c < heads % chunks ? 1 : 0);
+        const size_t off = (size_t)h0 * head_bytes, len = (size_t)n_heads * head_bytes;
+        const uint8_t *qh = (const uint8_t*)q_host + off, *kh = (const uint8_t*)k_host + off, *vh = (const uint8_t*)v_host + off;
+        uint8_t *qd = (uint8_t*)q_dev + off, *kd = (uint8_t*)k_dev + off, *vd = (uint8_t*)v_dev + off, *od = (uint8_t*)o_dev + off;
+        if ((e = cudaMemcpyAsync(qd, qh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(kd, kh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(vd, vh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess)
+            return fail_cuda("host-to-device copy");
+        if ((e = cudaEventRecord(hp->uploaded[c], hp->up)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->run, hp->uploaded[c], 0)) != cudaSuccess)
+            return fail_cuda("cudaEventRecord");
+        rc = attn_fwd_ex(qd, kd, vd, od, 1, (int)n_heads, N, d, scale, causal, scan_order, dtype, hp->run, opts);
+        if (rc) return rc;
+        if ((e = cudaEventRecord(hp->computed[c], hp->run)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->down, hp->computed[c], 0)) != cudaSuccess)
+            return fail_cuda("cudaEventRecord");
+        if ((e = cudaMemcpyAsync((uint8_t*)o_host + off, od, len, cudaMemcpyDeviceToHost, hp->down)) != cudaSuccess)
+            return fail_cuda("device-to-host copy");
+        h0 += n_heads;
     }
+    if ((e = cudaEventRecord(hp->done, hp->down)) != cudaSuccess || (e = cudaStreamWaitEvent(st, hp->done, 0)) != cudaSuccess)
+        return fail_cuda("cudaEventRecord");
     return ATTN_OK;
 }
 

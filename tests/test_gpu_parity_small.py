@@ -138,3 +138,29 @@ def test_bad_arguments_are_rejected_before_launch():
             sa.attn_fwd(a["q"], a["k"], a["v"], a["o"], a["B"], a["H"], a["N"], a["d"], a["scale"], a["causal"],
                         a["scan_order"], a["dtype"], st)
         assert e.value.status == status, (change, e.value)
+
+
+@pytest.mark.parametrize("host_chunks", [1, 3, 16])
+def test_host_entry_point_pipeline_matches_device_entry_point(host_chunks):
+    """attn_fwd_host (pinned host buffers in and out, heads cut into groups that are uploaded, computed and
+    downloaded as a pipeline) gives the device entry point's result bit for bit in the cyclic order."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("host", 1, 5, 700, 128, wl.BF16, True, 7350)
+    q, k, v = upload(w)
+    want = run_cuda(w, (q, k, v), sa.CYCLIC)
+    host = [t.view(torch.int16).cpu().pin_memory() for t in (q, k, v)]
+    o_host = torch.full(q.shape, -1, dtype=torch.int16).pin_memory()
+    dev = [torch.empty_like(q) for _ in range(4)]
+    opts = sa.Opts()
+    opts.host_chunks = host_chunks
+    stream = torch.cuda.Stream()
+    for _ in range(2):   # twice: the second call reuses the pipeline's events
+        o_host.fill_(-1)
+        sa.attn_fwd_host(host[0].data_ptr(), host[1].data_ptr(), host[2].data_ptr(), o_host.data_ptr(), dev[0].data_ptr(),
+                         dev[1].data_ptr(), dev[2].data_ptr(), dev[3].data_ptr(), w.B, w.H, w.N, w.d, w.scale, 1, sa.CYCLIC,
+                         sa.BF16, stream.cuda_stream, opts)
+        stream.synchronize()
+        sa.attn_device_status()
+        assert torch.equal(o_host, want.view(torch.int16).cpu())
+    assert_parity(w, o_host.view(torch.bfloat16).cuda())
