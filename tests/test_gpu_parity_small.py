@@ -164,3 +164,36 @@ def test_host_entry_point_pipeline_matches_device_entry_point(host_chunks):
         sa.attn_device_status()
         assert torch.equal(o_host, want.view(torch.int16).cpu())
     assert_parity(w, o_host.view(torch.bfloat16).cuda())
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_large_score_range_exercises_the_lazy_rescale(causal):
+    """K scaled by 8: scores spread over +-35 in log2 units, so the running maximum jumps by more than the rescale
+    threshold between tiles again and again, and the softmax is close to one-hot."""
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("peaky", 1, 3, 1500, 128, wl.BF16, causal, 7360, k_scale=8.0)
+    qkv = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        assert_parity(w, run_cuda(w, qkv, order))
+
+
+def test_monotonically_growing_scores_and_uniform_scores():
+    """Scores that grow with the key index (every tile raises the row maximum in a forward scan, none in a backward
+    one) and scores that are all equal (K = 0: O is the mean, or prefix mean, of V), against the oracle."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    from oracle import attention as ora
+    N, d = 1100, 64
+    g = torch.Generator(device="cpu").manual_seed(11)
+    v = torch.randn(1, 1, N, d, generator=g).to(torch.float16)
+    q = torch.full((1, 1, N, d), 0.5, dtype=torch.float16)
+    ramp = (torch.arange(N, dtype=torch.float32) * (1.0 / 16.0)).view(1, 1, N, 1).expand(1, 1, N, d).contiguous().to(torch.float16)
+    for k, causal in ((ramp, False), (ramp, True), (torch.zeros_like(q), True)):
+        want = ora.attention_head(q[0, 0].double().numpy(), k[0, 0].double().numpy(), v[0, 0].double().numpy(), 0.125, causal)
+        opts = sa.Opts()
+        opts.max_ctas = 2
+        for order in (sa.CYCLIC, sa.SAWTOOTH):
+            o = sa.forward(q.cuda(), k.cuda(), v.cuda(), causal=causal, scan_order=order, scale=0.125, opts=opts)
+            sa.attn_device_status()
+            err = np.abs(o[0, 0].double().cpu().numpy() - want)
+            assert err.max() <= 2e-2 and err.mean() <= 2e-3, (causal, order, err.max(), err.mean())
