@@ -381,8 +381,12 @@ def main():
     flops = w.flops
     ms_head = results[headline]
     tf_head = whole_job_tflops(flops, ms_head, 1)  # one GPU's throughput; `value` is the job's
+    # Which measured peak the run is compared with: the sustained one when the timed launches ran as one long,
+    # power-capped load (half a second or more of it, or the cap seen by NVML with the kernel's own clock under 80 % of
+    # the maximum), else the burst one.  Both fractions are in the line either way.
     timed_region_s = ms_head * args.steps / 1e3
-    peak_kind = "sustained" if timed_region_s >= 0.5 else "burst"
+    capped = "sw_power_cap" in clk.get("reasons", []) and clk.get("sm_max_mhz") and clk["kernel_mhz"] < 0.8 * clk["sm_max_mhz"]
+    peak_kind = "sustained" if (timed_region_s >= 0.5 or capped) else "burst"
     peak = peaks[peak_kind]
     plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt, run_opts)
     line = {
