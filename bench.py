@@ -202,6 +202,8 @@ def main():
     ap.add_argument("--scan-order", default="both", choices=["both", "cyclic", "sawtooth"],
                     help="orders to time; `value` is the sawtooth order unless only cyclic is timed")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--digit-order", default="tile", choices=["tile", "head"],
+                    help="which digit of the linear work index varies fastest: the Q block (default) or the head")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the persistent grid (the paper's 'active SMs'); 0 = all SMs")
     ap.add_argument("--also", default="c2,c4,c5",
                     help="further workloads timed briefly in both orders (single GPU only; '' for none)")
@@ -252,9 +254,10 @@ def main():
     sh = stream.cuda_stream
 
     run_opts = None
-    if args.max_ctas > 0:
+    if args.max_ctas > 0 or args.digit_order == "head":
         run_opts = sa.Opts()
         run_opts.max_ctas = args.max_ctas
+        run_opts.digit_order = sa.HEAD_FASTEST if args.digit_order == "head" else sa.TILE_FASTEST
 
     def make_step(bufs, wk, a_dt):
         def step(order):
