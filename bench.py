@@ -221,9 +221,12 @@ def main():
 
     import torch
     import paper_2601_16032_b200 as sa
+    from paper_2601_16032_b200 import build as lib_build
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        lib_build.build()  # compiles the CUDA library in-tree if it is missing or older than its sources
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

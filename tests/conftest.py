@@ -15,3 +15,12 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """The C-ABI library and the C part of the oracle are built in-tree before any test (a no-op when they are fresh)."""
+    from paper_2601_16032_b200 import build as lib_build
+    from oracle import build as oracle_build
+    lib_build.build()
+    oracle_build.build()
