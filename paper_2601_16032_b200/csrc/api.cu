@@ -128,18 +128,20 @@ int get_encoder(EncodeTiledFn* fn) {
     return ATTN_OK;
 }
 
-// [B*H, N, d] view, box = 64 columns x `rows` rows of one head, 128-byte swizzle, zero fill outside.
-int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype) {
+// [B*H, N, d] view, box = `cols` (64 or 32) columns x `rows` rows of one head, rows of the box swizzled over their
+// own length (128 or 64 bytes), zero fill outside.
+int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype, int cols = 64) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc) return rc;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)cols, (cuuint32_t)rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(m, dtype == ATTN_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
     return ATTN_OK;
 }
@@ -214,7 +216,7 @@ int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const att
     out->items_per_head = sp.n_q;
     out->n_work = sp.n_work;
     out->grid = grid_for(sp.n_work, sm_count, r);
-    out->threads = r.q_tiles * 128 * SAW_THREADS_PER_ROW + 128;
+    out->threads = 384;  // eight softmax warps, the producer warp, two MMA warps, one idle warp
     out->kv_stages = r.stages;
     out->smem_bytes = (int)r.smem;
     out->sm_count = sm_count;
@@ -334,10 +336,12 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
     if ((rc = make_map(&tq, q, B * H, N, d, kBlockM, dtype))) return rc;
     if ((rc = make_map(&tk, k, B * H, N, d, r.block_n, dtype))) return rc;
     if ((rc = make_map(&tv, v, B * H, N, d, r.block_n, dtype))) return rc;
-    // O is written through shared memory in boxes of 64 columns x as many rows as one warp's share of a ring slot holds.
+    // O is written through shared memory, each softmax warp storing boxes of its d/2 columns x as many rows (at most its
+    // 32) as its eighth of a ring slot holds.
     CUtensorMap to;
-    const int stage_rows = (r.block_n * d * 2 / 2 / 4) / 128 < 32 ? (r.block_n * d * 2 / 2 / 4) / 128 : 32;
-    if ((rc = make_map(&to, o, B * H, N, d, stage_rows, dtype))) return rc;
+    const int stage_row_bytes = d, stage_bytes_per_warp = r.block_n * d * 2 / 8;
+    const int stage_rows = stage_bytes_per_warp / stage_row_bytes < 32 ? stage_bytes_per_warp / stage_row_bytes : 32;
+    if ((rc = make_map(&to, o, B * H, N, d, stage_rows, dtype, d / 2))) return rc;
 
     const int grid = grid_for(kp.sched.n_work, sm_count, r);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
