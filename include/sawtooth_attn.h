@@ -21,7 +21,8 @@
  * all of the same type (IEEE fp16 or bfloat16); N_q = N_k = N.  Products accumulate in fp32; the
  * probabilities are rounded to the 16-bit type before the second product; O is rounded once at the
  * end.  Supported: d in {64, 128}; any B, H, N >= 1 with B*H <= 2^31-1 and N <= 2^24; scale finite
- * and > 0.  Every base pointer must be 16-byte aligned.  `o` must not overlap q, k or v.
+ * (any sign; zero gives every visible key the same weight).  Every base pointer must be 16-byte aligned.  `o` must
+ * not overlap q, k or v.
  *
  * Ownership: the caller owns every buffer; the library allocates no device memory.  Calls enqueue
  * work on the given stream and return without waiting (except where stated).  For fixed arguments
@@ -53,6 +54,18 @@ typedef enum {
 typedef enum { ATTN_SCAN_CYCLIC = 0, ATTN_SCAN_SAWTOOTH = 1 } attn_scan_order;
 typedef enum { ATTN_F16 = 0, ATTN_BF16 = 1 } attn_dtype;
 typedef enum { ATTN_TILE_FASTEST = 0, ATTN_HEAD_FASTEST = 1 } attn_digit_order;
+/*
+ * How the static walk of Algorithm 2 groups work items.  With pairs, a unit of the walk is two W-row Q blocks of one
+ * head which the CTA handles one after the other, the first scanned first-to-last and, in the sawtooth order, the
+ * second last-to-first: the form with two Q tiles per loop trip that the paper's tile-based kernels use.
+ *   ATTN_PAIR_MIRRORED  blocks (n-1-p, p) of a head with n blocks.  Under the causal mask block q scans q+1 blocks' worth
+ *                       of K/V tiles, so every pair scans n+1: all units take the same time, the static walk is balanced,
+ *                       the CTAs of a wave stay in step and, in the sawtooth order, read the same two K/V tiles at any time.
+ *   ATTN_PAIR_ADJACENT  blocks (2p, 2p+1).
+ *   ATTN_PAIR_NONE      one block per unit (Algorithm 2 as printed).
+ *   ATTN_PAIR_DEFAULT   mirrored under the causal mask, none otherwise.  The dynamic schedule never pairs.
+ */
+typedef enum { ATTN_PAIR_DEFAULT = 0, ATTN_PAIR_NONE = 1, ATTN_PAIR_MIRRORED = 2, ATTN_PAIR_ADJACENT = 3 } attn_pairing;
 
 /* Optional knobs; zero-initialise, then set what you need.  0 always means "library default". */
 typedef struct {
@@ -64,7 +77,13 @@ typedef struct {
     int launch_mode;  /* 0: persistent grid (Algorithm 2); 1: one CTA per work item (Algorithm 3) */
     int l2_policy;    /* 0: no hint; 1: K/V loads carry an evict_last hint, Q loads evict_first */
     int host_chunks;  /* attn_fwd_host only: pieces the heads are cut into so that copies and kernels overlap (1..16; 0 = automatic) */
-    int reserved[8];
+    float* lse;       /* optional DEVICE output [B, H, N] (fp32, 4-byte aligned), NULL for none: per query row the natural log of
+                         the softmax denominator, ln sum_j exp(scale * q_i . k_j) over the keys the row may see (the quantity a
+                         backward pass or a merge of partial results needs; outside the paper).  Ignored by attn_fwd_host. */
+    int pairing;      /* attn_pairing: whether one trip of a CTA's loop takes one work item or a pair of them (see below) */
+    int check_mode;   /* 1: the call waits for the device and returns ATTN_ERR_DEVICE_TIMEOUT itself if a bounded wait inside
+                         its kernel (or an earlier one on the device) ran out; 0: asynchronous, poll attn_device_status */
+    int reserved[4];
 } attn_fwd_opts;
 
 /* What a call with these arguments will launch; lets a caller predict L2 traffic. */
@@ -80,18 +99,21 @@ typedef struct {
     int kv_stages;      /* ring slots (each holds one K tile or one V tile) */
     int smem_bytes;     /* dynamic shared memory per CTA */
     int sm_count;       /* SMs of the device the plan was made for */
+    int pairing;        /* attn_pairing in force (never ATTN_PAIR_DEFAULT) */
+    long long n_units;  /* units of the static walk: n_work, or B * H * ceil(items_per_head / 2) with pairs; grid = min(n_units, SMs) */
 } attn_plan;
 
 /* One work item as a CTA handles it (host-side replay of the device schedule). */
 typedef struct {
     int cta;            /* blockIdx.x */
-    int iteration;      /* the CTA's local iteration count (Algorithm 4's i_local) */
-    long long k;        /* linear work index */
+    int iteration;      /* the CTA's count of items handled so far (Algorithm 4's i_local) */
+    long long k;        /* linear index of the unit the walk is at (k = cta, += grid); with pairs two entries share one k */
     int batch, head;
     int q_item;         /* index of the W-row block inside the head */
     int backward;       /* 1: K/V tiles scanned last to first */
     int n_kv;           /* tiles 0 .. n_kv-1 are scanned */
     int n_kv_q0, n_kv_q1; /* of those, the ones the first / second 128-row Q tile takes part in */
+    int member;         /* 0 or 1: which item of its pair this is (0 without pairs) */
 } attn_trace_entry;
 
 /*
@@ -117,7 +139,8 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o,
  * backward depends on the race for the counter: results are reproducible bit for bit in the cyclic order only.
  *
  * scratch: DEVICE memory owned by the caller, 4-byte aligned, at least attn_dynamic_scratch_bytes(plan.grid) bytes
- * (plan from attn_query_plan; ATTN_DYNAMIC_SCRATCH_HEADER + 4 bytes per CTA).  The call clears it on `stream` before
+ * (plan from attn_query_plan with opts->pairing = ATTN_PAIR_NONE, since single items are claimed here;
+ * ATTN_DYNAMIC_SCRATCH_HEADER + 4 bytes per CTA; the SM count of the device is always enough).  The call clears it on `stream` before
  * the kernel; afterwards int[0] holds the number of claims made and int[64 + c] the number of items CTA c handled.
  * Two calls that share one scratch buffer must not overlap on the GPU.  launch_mode must be 0.
  */

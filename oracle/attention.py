@@ -1,6 +1,7 @@
 """fp64 attention oracle (test infrastructure; the CUDA path never touches it).
 
-Three statements of the same result:
+Three statements of the same result (and, beside them, the logarithm of the softmax denominator per row,
+`logsumexp_definition` / `logsumexp_rows`, which the CUDA path can emit as a second output):
 
 * `attention_definition` -- Eq. 1 written out with numpy: the full N x N score matrix, a row
   softmax, a product with V.  It is the reference for small cases.
@@ -35,6 +36,11 @@ def _c():
         lib.attn_ref_rows.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+            ctypes.c_double, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+        ]
+        lib.attn_ref_lse_rows.restype = ctypes.c_int
+        lib.attn_ref_lse_rows.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
             ctypes.c_double, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
         ]
         lib.attn_ref_threads.restype = ctypes.c_int
@@ -78,6 +84,37 @@ def attention_rows(q_rows: np.ndarray, row_index: np.ndarray, k: np.ndarray, v: 
                             N, d, float(scale), int(bool(causal)), int(threads), out.ctypes.data)
     if rc != 0:
         raise RuntimeError(f"attn_ref_rows failed ({rc})")
+    return out
+
+
+def logsumexp_definition(q: np.ndarray, k: np.ndarray, scale: float, causal: bool) -> np.ndarray:
+    """ln of Eq. 1's softmax denominator per query row: ln sum_j exp(scale * q_i . k_j) over the visible keys."""
+    q = np.asarray(q, np.float64)
+    k = np.asarray(k, np.float64)
+    s = scale * (q @ k.T)
+    if causal:
+        i = np.arange(q.shape[0])[:, None]
+        j = np.arange(k.shape[0])[None, :]
+        s = np.where(j <= i, s, -np.inf)
+    m = s.max(axis=1)
+    return m + np.log(np.exp(s - m[:, None]).sum(axis=1))
+
+
+def logsumexp_rows(q_rows: np.ndarray, row_index: np.ndarray, k: np.ndarray, scale: float, causal: bool,
+                   threads: int = 0) -> np.ndarray:
+    """The same per-row logarithm for chosen query rows of one head, via attn_ref.c."""
+    q_rows = np.ascontiguousarray(q_rows, np.float64)
+    row_index = np.ascontiguousarray(row_index, np.int64)
+    k = np.ascontiguousarray(k, np.float64)
+    n_rows, d = q_rows.shape
+    N = k.shape[0]
+    if k.shape != (N, d) or row_index.shape != (n_rows,):
+        raise ValueError("shape mismatch")
+    out = np.empty(n_rows, np.float64)
+    rc = _c().attn_ref_lse_rows(q_rows.ctypes.data, row_index.ctypes.data, n_rows, k.ctypes.data, N, d, float(scale),
+                                int(bool(causal)), int(threads), out.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"attn_ref_lse_rows failed ({rc})")
     return out
 
 

@@ -86,3 +86,52 @@ int attn_ref_rows(const double *q_rows, const int64_t *row_index, int64_t n_rows
     }
     return failed ? -1 : 0;
 }
+
+/*
+ * The softmax denominator of the same definition, as a logarithm: for query row i,
+ *
+ *     lse[i] = ln sum_j exp(s_j) = max_j s_j + ln sum_j exp(s_j - max_j s_j),   s_j = scale * q[i,:] . k[j,:]
+ *
+ * over the keys the row may see.  (Not in the paper: it is the per-row quantity a backward pass or a merge of
+ * partial attention results needs, and the CUDA path can emit it.)  Arguments as attn_ref_rows; out: [n_rows].
+ */
+int attn_ref_lse_rows(const double *q_rows, const int64_t *row_index, int64_t n_rows,
+                      const double *k, int64_t N, int64_t d, double scale, int causal, int threads, double *out)
+{
+    if (!q_rows || !row_index || !k || !out || n_rows < 0 || N <= 0 || d <= 0) return -1;
+    for (int64_t r = 0; r < n_rows; ++r)
+        if (row_index[r] < 0 || row_index[r] >= N) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (threads > 0) omp_set_num_threads(threads);
+#else
+    (void)threads;
+#endif
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)N * sizeof(double));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            if (!s) continue;
+            const double *qi = q_rows + r * d;
+            const int64_t visible = causal ? row_index[r] + 1 : N;
+            double smax = -INFINITY;
+            for (int64_t j = 0; j < visible; ++j) {
+                const double *kj = k + j * d;
+                double dot = 0.0;
+                for (int64_t t = 0; t < d; ++t) dot += qi[t] * kj[t];
+                s[j] = scale * dot;
+                if (s[j] > smax) smax = s[j];
+            }
+            double denom = 0.0;
+            for (int64_t j = 0; j < visible; ++j) denom += exp(s[j] - smax);
+            out[r] = smax + log(denom);
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}

@@ -13,6 +13,15 @@ first.  The cyclic order always scans from the first to the last.
 
 Causal mask: Q tile t (rows t*W .. min(N,(t+1)*W)-1) needs K/V tiles 0 .. hi-1 with
 hi = ceil(min(N,(t+1)*W) / B_c); the tiles beyond are never visited, in either direction.
+
+Pairs (the tile-based form of the sawtooth, where one trip of the persistent loop takes two Q tiles, the
+first scanned forward and the second backward): with pairing the units that Algorithm 2's walk
+hands out are pairs of Q tiles of one head, handled one after the other by the same CTA.
+"adjacent" pairs are (2p, 2p+1).  "mirrored" pairs are (n_q-1-p, p): under the causal mask tile t
+scans about t+1 tiles' worth of K/V, so the two members of a mirrored pair scan n_q+1 between them
+whatever p is, and all units take the same time.  An odd middle tile forms a unit of its own.
+i_local still counts Q tiles, so in the sawtooth order the first member of a pair is scanned
+forward and the second backward.
 """
 from __future__ import annotations
 
@@ -33,6 +42,7 @@ class WorkItem:
     q_tile: int
     backward: bool
     n_kv: int  # K/V tiles this Q tile visits (0 .. n_kv-1)
+    member: int = 0  # which Q tile of its pair this is (0 without pairing)
 
     def kv_order(self) -> range:
         return range(self.n_kv - 1, -1, -1) if self.backward else range(self.n_kv)
@@ -69,23 +79,42 @@ def kv_tiles_needed(t: int, N: int, W: int, B_c: int, causal: bool) -> int:
     return ceil_div(last_row_excl, B_c)
 
 
+def unit_members(p: int, n_q: int, pairing: str) -> list[int]:
+    """The Q tiles of a head that unit p of the walk holds, in the order the CTA handles them."""
+    if pairing == "none":
+        return [p]
+    if pairing == "mirrored":
+        far, near = n_q - 1 - p, p
+        return [far] if far == near else [far, near]
+    if pairing == "adjacent":
+        return [t for t in (2 * p, 2 * p + 1) if t < n_q]
+    raise ValueError(pairing)
+
+
+def units_per_head(n_q: int, pairing: str) -> int:
+    return n_q if pairing == "none" else ceil_div(n_q, 2)
+
+
 def cta_sequence(cta: int, G: int, B: int, H: int, N: int, W: int, B_c: int, causal: bool,
-                 scan_order: int, digit_order: str = "tile_fastest") -> Iterator[WorkItem]:
+                 scan_order: int, digit_order: str = "tile_fastest", pairing: str = "none") -> Iterator[WorkItem]:
     """The Q tiles one CTA handles, in order, each with its K/V scan (Algorithms 2 and 4)."""
     n_q = ceil_div(N, W)
-    n_tiles = B * H * n_q
+    n_u = units_per_head(n_q, pairing)
+    n_units = B * H * n_u
     i_local = 0
     k = cta
-    while k < n_tiles:
-        b, h, t = decode(k, B, H, n_q, digit_order)
-        backward = scan_order == SAWTOOTH and i_local % 2 == 1
-        yield WorkItem(cta, i_local, k, b, h, t, backward, kv_tiles_needed(t, N, W, B_c, causal))
-        i_local += 1
+    while k < n_units:
+        b, h, p = decode(k, B, H, n_u, digit_order)
+        for member, t in enumerate(unit_members(p, n_q, pairing)):
+            backward = scan_order == SAWTOOTH and i_local % 2 == 1
+            yield WorkItem(cta, i_local, k, b, h, t, backward, kv_tiles_needed(t, N, W, B_c, causal), member)
+            i_local += 1
         k += G
 
 
 def full_schedule(n_sm: int, B: int, H: int, N: int, W: int, B_c: int, causal: bool,
-                  scan_order: int, digit_order: str = "tile_fastest", max_ctas: int = 0) -> list[list[WorkItem]]:
-    n_tiles = B * H * ceil_div(N, W)
-    G = grid_size(n_tiles, n_sm if max_ctas <= 0 else min(n_sm, max_ctas))
-    return [list(cta_sequence(c, G, B, H, N, W, B_c, causal, scan_order, digit_order)) for c in range(G)]
+                  scan_order: int, digit_order: str = "tile_fastest", max_ctas: int = 0,
+                  pairing: str = "none") -> list[list[WorkItem]]:
+    n_units = B * H * units_per_head(ceil_div(N, W), pairing)
+    G = grid_size(n_units, n_sm if max_ctas <= 0 else min(n_sm, max_ctas))
+    return [list(cta_sequence(c, G, B, H, N, W, B_c, causal, scan_order, digit_order, pairing)) for c in range(G)]

@@ -8,6 +8,7 @@ from typing import Optional
 CYCLIC, SAWTOOTH = 0, 1
 F16, BF16 = 0, 1
 TILE_FASTEST, HEAD_FASTEST = 0, 1
+PAIR_DEFAULT, PAIR_NONE, PAIR_MIRRORED, PAIR_ADJACENT = 0, 1, 2, 3
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libsawtooth_attn.so")
@@ -25,7 +26,8 @@ class Opts(ctypes.Structure):
     _fields_ = [
         ("max_ctas", ctypes.c_int), ("kv_stages", ctypes.c_int), ("block_n", ctypes.c_int),
         ("q_tiles", ctypes.c_int), ("digit_order", ctypes.c_int), ("launch_mode", ctypes.c_int),
-        ("l2_policy", ctypes.c_int), ("host_chunks", ctypes.c_int), ("reserved", ctypes.c_int * 8),
+        ("l2_policy", ctypes.c_int), ("host_chunks", ctypes.c_int), ("lse", ctypes.c_void_p), ("pairing", ctypes.c_int), ("check_mode", ctypes.c_int),
+        ("reserved", ctypes.c_int * 4),
     ]
 
 
@@ -34,7 +36,7 @@ class Plan(ctypes.Structure):
         ("block_m", ctypes.c_int), ("block_n", ctypes.c_int), ("q_tiles", ctypes.c_int),
         ("rows_per_item", ctypes.c_int), ("items_per_head", ctypes.c_int), ("n_work", ctypes.c_longlong),
         ("grid", ctypes.c_int), ("threads", ctypes.c_int), ("kv_stages", ctypes.c_int),
-        ("smem_bytes", ctypes.c_int), ("sm_count", ctypes.c_int),
+        ("smem_bytes", ctypes.c_int), ("sm_count", ctypes.c_int), ("pairing", ctypes.c_int), ("n_units", ctypes.c_longlong),
     ]
 
 
@@ -43,6 +45,7 @@ class TraceEntry(ctypes.Structure):
         ("cta", ctypes.c_int), ("iteration", ctypes.c_int), ("k", ctypes.c_longlong),
         ("batch", ctypes.c_int), ("head", ctypes.c_int), ("q_item", ctypes.c_int),
         ("backward", ctypes.c_int), ("n_kv", ctypes.c_int), ("n_kv_q0", ctypes.c_int), ("n_kv_q1", ctypes.c_int),
+        ("member", ctypes.c_int),
     ]
 
 

@@ -31,14 +31,28 @@ __device__ unsigned long long g_cycles = 0;
 // Scratch of attn_fwd_dynamic_noalloc: the claim counter block and one counter per CTA, resident in every GPU
 // that loads the library for as long as the process lives.
 static __device__ __align__(256) int g_noalloc_scratch[(ATTN_DYNAMIC_SCRATCH_HEADER / 4) + ATTN_NOALLOC_MAX_CTAS];
-constexpr int kMaxDevices = 64;
-int* g_noalloc_ptr[kMaxDevices] = {};  // device address of the array above, per device, once looked up
 
+constexpr int kMaxDevices = 64;
 constexpr int kMaxHostChunks = 16;
 constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
+constexpr int kKernelVariants = 16;     // d x block_n x q_tiles x dtype
+
+// What the library knows about a device, looked up once (under the mutex) on the first call that has it current:
+// its size, the device addresses of the library's own __device__ variables there, and which kernel variants have had
+// their dynamic shared memory limit raised.  Readers take a copy under the same mutex.
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0, smem_optin = 0;
+    int* status = nullptr;
+    unsigned long long* cycles = nullptr;
+    int* noalloc_scratch = nullptr;
+    unsigned smem_raised = 0;   // bit v: variant v of the kernel may use smem_optin bytes
+};
+DeviceState g_device[kMaxDevices];
+std::mutex g_device_mutex;
 
 struct Resolved {
-    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas;
+    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas, pairing, check_mode;
     size_t smem;
 };
 
@@ -56,7 +70,8 @@ int check_shape(int B, int H, int N, int d, int causal, int dtype) {
     return ATTN_OK;
 }
 
-int resolve_opts(const attn_fwd_opts* o, int d, int smem_limit, Resolved* r) {
+// `dynamic`: the call uses the dynamic schedule (items are claimed one by one, so there are no pairs).
+int resolve_opts(const attn_fwd_opts* o, int d, int causal, bool dynamic, int smem_limit, Resolved* r) {
     attn_fwd_opts z;
     memset(&z, 0, sizeof(z));
     if (o) z = *o;
@@ -70,6 +85,14 @@ int resolve_opts(const attn_fwd_opts* o, int d, int smem_limit, Resolved* r) {
     if (z.l2_policy != 0 && z.l2_policy != 1) return fail(ATTN_ERR_INVALID_ARG, "l2_policy must be 0 or 1");
     if (z.max_ctas < 0 || z.kv_stages < 0) return fail(ATTN_ERR_INVALID_ARG, "max_ctas and kv_stages must be >= 0");
     if (z.host_chunks < 0 || z.host_chunks > kMaxHostChunks) return fail(ATTN_ERR_INVALID_ARG, "host_chunks must be in [0, %d]", kMaxHostChunks);
+    if (z.pairing < ATTN_PAIR_DEFAULT || z.pairing > ATTN_PAIR_ADJACENT) return fail(ATTN_ERR_INVALID_ARG, "unknown pairing %d", z.pairing);
+    if (z.check_mode != 0 && z.check_mode != 1) return fail(ATTN_ERR_INVALID_ARG, "check_mode must be 0 or 1");
+    if (dynamic && z.pairing > ATTN_PAIR_NONE) return fail(ATTN_ERR_INVALID_ARG, "the dynamic schedule claims single work items: pairing must be left at its default or be ATTN_PAIR_NONE");
+    // Default: mirrored pairs under the causal mask (every unit of the static walk then takes the same time), none otherwise.
+    r->pairing = dynamic ? kPairNone
+               : z.pairing == ATTN_PAIR_DEFAULT ? (causal ? kPairMirrored : kPairNone)
+               : z.pairing == ATTN_PAIR_NONE ? kPairNone : z.pairing == ATTN_PAIR_MIRRORED ? kPairMirrored : kPairAdjacent;
+    r->check_mode = z.check_mode;
     r->head_fastest = z.digit_order == ATTN_HEAD_FASTEST;
     r->launch_mode = z.launch_mode;
     r->l2_policy = z.l2_policy;
@@ -88,24 +111,43 @@ int resolve_opts(const attn_fwd_opts* o, int d, int smem_limit, Resolved* r) {
     return ATTN_OK;
 }
 
-int device_sm_count(int* sms, int* smem_optin) {
+// The current device's entry of g_device, filled on first use.  *dev_out gets the device index.
+int current_device(DeviceState* out, int* dev_out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
-    int major = 0;
-    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
-    if (major != 10) return fail(ATTN_ERR_UNSUPPORTED, "device compute capability %d.x is not 10.x", major);
-    cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device index %d is beyond the %d the library keeps track of", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    DeviceState& ds = g_device[dev];
+    if (!ds.ready) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
+        if (major != 10) return fail(ATTN_ERR_UNSUPPORTED, "device compute capability %d.x is not 10.x", major);
+        cudaDeviceGetAttribute(&ds.sm_count, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&ds.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        // In host code the names of __device__ variables are only handles for this lookup, not addresses a kernel could
+        // use; the lookup gives the address inside the current device.
+        if ((e = cudaGetSymbolAddress((void**)&ds.status, g_status_word)) != cudaSuccess ||
+            (e = cudaGetSymbolAddress((void**)&ds.cycles, g_cycles)) != cudaSuccess ||
+            (e = cudaGetSymbolAddress((void**)&ds.noalloc_scratch, g_noalloc_scratch)) != cudaSuccess ||
+            !ds.status || !ds.cycles || !ds.noalloc_scratch) {
+            cudaGetLastError();
+            return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        }
+        ds.ready = true;
+    }
+    *out = ds;
+    if (dev_out) *dev_out = dev;
     return ATTN_OK;
 }
 
-int grid_for(long long n_work, int sm_count, const Resolved& r) {
+// n_units: work items, or pairs of them (what one trip of a CTA's loop handles).
+int grid_for(long long n_units, int sm_count, const Resolved& r) {
     long long cap = sm_count;
     if (r.max_ctas > 0 && r.max_ctas < cap) cap = r.max_ctas;
-    if (r.launch_mode == 1) return (int)(n_work < 2147483647LL ? n_work : 2147483647LL);  // Algorithm 3
-    return (int)(n_work < cap ? n_work : cap);                                           // Algorithm 2
+    if (r.launch_mode == 1) return (int)(n_units < 2147483647LL ? n_units : 2147483647LL);  // Algorithm 3
+    return (int)(n_units < cap ? n_units : cap);                                            // Algorithm 2
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -128,52 +170,104 @@ int get_encoder(EncodeTiledFn* fn) {
     return ATTN_OK;
 }
 
-// [B*H, N, d] view, box = `cols` (64 or 32) columns x `rows` rows of one head, rows of the box swizzled over their
-// own length (128 or 64 bytes), zero fill outside.
-int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype, int cols = 64) {
+// [B*H, N, d] view, box = 64 columns x `rows` rows of one head, 128-byte swizzle, zero fill outside.
+int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc) return rc;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {(cuuint32_t)cols, (cuuint32_t)rows, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(m, dtype == ATTN_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
     return ATTN_OK;
 }
 
+// The four tensor maps of a call are a pure function of (pointers, shape, type, tile shape); the last few a host
+// thread built are kept, so that a caller who launches on the same buffers again and again pays for the encoding once.
+struct MapKey {
+    const void *q, *k, *v, *o;
+    int BH, N, d, dtype, block_n, stage_rows;
+    bool operator==(const MapKey& x) const {
+        return q == x.q && k == x.k && v == x.v && o == x.o && BH == x.BH && N == x.N && d == x.d && dtype == x.dtype &&
+               block_n == x.block_n && stage_rows == x.stage_rows;
+    }
+};
+struct MapSet { MapKey key; CUtensorMap tq, tk, tv, to; bool valid = false; };
+constexpr int kMapCacheSize = 8;
+thread_local MapSet g_maps[kMapCacheSize];
+thread_local int g_maps_next = 0;
+
+int maps_for(const MapKey& key, const MapSet** out) {
+    for (int i = 0; i < kMapCacheSize; ++i)
+        if (g_maps[i].valid && g_maps[i].key == key) { *out = &g_maps[i]; return ATTN_OK; }
+    MapSet& m = g_maps[g_maps_next];
+    m.valid = false;
+    int rc;
+    if ((rc = make_map(&m.tq, key.q, key.BH, key.N, key.d, kBlockM, key.dtype))) return rc;
+    if ((rc = make_map(&m.tk, key.k, key.BH, key.N, key.d, key.block_n, key.dtype))) return rc;
+    if ((rc = make_map(&m.tv, key.v, key.BH, key.N, key.d, key.block_n, key.dtype))) return rc;
+    // O is written through shared memory in boxes of 64 columns x as many rows as one warp's share of a ring slot holds.
+    if ((rc = make_map(&m.to, key.o, key.BH, key.N, key.d, key.stage_rows, key.dtype))) return rc;
+    m.key = key;
+    m.valid = true;
+    g_maps_next = (g_maps_next + 1) % kMapCacheSize;
+    *out = &m;
+    return ATTN_OK;
+}
+
 template <int kD, int kBlockN, int kQTiles, int kBf16>
-int launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const KernelParams& kp, int grid,
-           size_t smem, cudaStream_t stream) {
+int launch(int dev, const DeviceState& ds, const MapSet& m, const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
     auto kern = attn_fwd_kernel<kD, kBlockN, kQTiles, kBf16>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); }
-    kern<<<grid, Geometry<kD, kBlockN, kQTiles>::kThreads, smem, stream>>>(tq, tk, tv, to, kp);
-    e = cudaGetLastError();
+    constexpr int variant = ((kD == 128) << 3) | ((kBlockN == 128) << 2) | ((kQTiles == 2) << 1) | kBf16;
+    static_assert(variant < kKernelVariants, "variant index");
+    if (!(ds.smem_raised & (1u << variant))) {
+        // Once per device and kernel variant: allow the kernel the device's whole opt-in shared memory.
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ds.smem_optin);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); }
+        std::lock_guard<std::mutex> lock(g_device_mutex);
+        g_device[dev].smem_raised |= 1u << variant;
+    }
+    kern<<<grid, Geometry<kD, kBlockN, kQTiles>::kThreads, smem, stream>>>(m.tq, m.tk, m.tv, m.to, kp);
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ATTN_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
     return ATTN_OK;
 }
 
 template <int kD, int kBlockN, int kQTiles>
-int launch_dtype(int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const KernelParams& kp,
-                 int grid, size_t smem, cudaStream_t stream) {
-    return dtype == ATTN_BF16 ? launch<kD, kBlockN, kQTiles, 1>(tq, tk, tv, to, kp, grid, smem, stream)
-                              : launch<kD, kBlockN, kQTiles, 0>(tq, tk, tv, to, kp, grid, smem, stream);
+int launch_dtype(int dtype, int dev, const DeviceState& ds, const MapSet& m, const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
+    return dtype == ATTN_BF16 ? launch<kD, kBlockN, kQTiles, 1>(dev, ds, m, kp, grid, smem, stream)
+                              : launch<kD, kBlockN, kQTiles, 0>(dev, ds, m, kp, grid, smem, stream);
 }
 
 template <int kD>
-int launch_tiles(int block_n, int q_tiles, int dtype, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                 const CUtensorMap& to, const KernelParams& kp, int grid, size_t smem, cudaStream_t stream) {
+int launch_tiles(int block_n, int q_tiles, int dtype, int dev, const DeviceState& ds, const MapSet& m, const KernelParams& kp, int grid,
+                 size_t smem, cudaStream_t stream) {
     if (block_n == 128) {
-        return q_tiles == 2 ? launch_dtype<kD, 128, 2>(dtype, tq, tk, tv, to, kp, grid, smem, stream)
-                            : launch_dtype<kD, 128, 1>(dtype, tq, tk, tv, to, kp, grid, smem, stream);
+        return q_tiles == 2 ? launch_dtype<kD, 128, 2>(dtype, dev, ds, m, kp, grid, smem, stream)
+                            : launch_dtype<kD, 128, 1>(dtype, dev, ds, m, kp, grid, smem, stream);
     }
-    return q_tiles == 2 ? launch_dtype<kD, 64, 2>(dtype, tq, tk, tv, to, kp, grid, smem, stream)
-                        : launch_dtype<kD, 64, 1>(dtype, tq, tk, tv, to, kp, grid, smem, stream);
+    return q_tiles == 2 ? launch_dtype<kD, 64, 2>(dtype, dev, ds, m, kp, grid, smem, stream)
+                        : launch_dtype<kD, 64, 1>(dtype, dev, ds, m, kp, grid, smem, stream);
+}
+
+// Reads and clears the current device's status word after a device synchronisation.
+int read_status(int* code) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e)); }
+    int word = 0;
+    e = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int));
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "reading the status word: %s", cudaGetErrorString(e)); }
+    if (code) *code = word;
+    if (word != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int));
+        return fail(ATTN_ERR_DEVICE_TIMEOUT, "kernel wait site %d ran out of time", word);
+    }
+    return ATTN_OK;
 }
 
 }  // namespace
@@ -202,24 +296,29 @@ int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const att
     if (rc) return rc;
     int smem_limit = kSmemOptinB200;
     if (sm_count <= 0) {
-        rc = device_sm_count(&sm_count, &smem_limit);
+        DeviceState ds;
+        rc = current_device(&ds, nullptr);
         if (rc) return rc;
+        sm_count = ds.sm_count;
+        smem_limit = ds.smem_optin;
     }
     Resolved r;
-    rc = resolve_opts(opts, d, smem_limit, &r);
+    rc = resolve_opts(opts, d, causal, false, smem_limit, &r);
     if (rc) return rc;
-    const SchedParams sp = make_sched(B, H, N, r.q_tiles, r.block_n, causal, 0, r.head_fastest);
+    const SchedParams sp = make_sched(B, H, N, r.q_tiles, r.block_n, causal, 0, r.head_fastest, 0, r.pairing);
     out->block_m = kBlockM;
     out->block_n = r.block_n;
     out->q_tiles = r.q_tiles;
     out->rows_per_item = kBlockM * r.q_tiles;
     out->items_per_head = sp.n_q;
     out->n_work = sp.n_work;
-    out->grid = grid_for(sp.n_work, sm_count, r);
-    out->threads = 384;  // eight softmax warps, the producer warp, two MMA warps, one idle warp
+    out->grid = grid_for(sp.n_units, sm_count, r);
+    out->threads = r.q_tiles * 128 + 128;
     out->kv_stages = r.stages;
     out->smem_bytes = (int)r.smem;
     out->sm_count = sm_count;
+    out->pairing = r.pairing == kPairNone ? ATTN_PAIR_NONE : r.pairing == kPairMirrored ? ATTN_PAIR_MIRRORED : ATTN_PAIR_ADJACENT;
+    out->n_units = sp.n_units;
     return ATTN_OK;
 }
 
@@ -233,17 +332,22 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
     int rc = attn_query_plan(B, H, N, d, causal, dtype, opts, sm_count, &plan);
     if (rc) return rc;
     const int head_fastest = opts && opts->digit_order == ATTN_HEAD_FASTEST;
-    const SchedParams sp = make_sched(B, H, N, plan.q_tiles, plan.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, head_fastest);
+    const int pairing = plan.pairing == ATTN_PAIR_NONE ? kPairNone : plan.pairing == ATTN_PAIR_MIRRORED ? kPairMirrored : kPairAdjacent;
+    const SchedParams sp = make_sched(B, H, N, plan.q_tiles, plan.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, head_fastest, 0, pairing);
+    const int members = pairing == kPairNone ? 1 : 2;
     size_t count = 0;
     for (int cta = 0; cta < plan.grid; ++cta) {
         int it = 0;
-        for (long long k = cta; k < sp.n_work; k += plan.grid, ++it) {
+        for (int slot = 0;; ++slot) {
+            const Slot sl = static_slot(sp, cta, plan.grid, slot);
+            if (sl.kind == kSlotEnd) break;
+            if (sl.kind == kSlotEmpty) continue;
             if (count < cap) {
-                const WorkItem w = decode_work(sp, k, it);
+                const WorkItem w = make_item(sp, sl.bh, sl.q_item, it);
                 attn_trace_entry* e = &buf[count];
                 e->cta = cta;
                 e->iteration = it;
-                e->k = k;
+                e->k = (long long)cta + (long long)(slot / members) * plan.grid;
                 e->batch = w.bh / H;
                 e->head = w.bh % H;
                 e->q_item = w.q_item;
@@ -251,8 +355,10 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
                 e->n_kv = w.hi;
                 e->n_kv_q0 = w.hi_q[0];
                 e->n_kv_q1 = w.hi_q[1];
+                e->member = slot % members;
             }
             ++count;
+            ++it;
         }
     }
     *n = count;
@@ -282,68 +388,71 @@ int attn_fwd_dynamic(const void* q, const void* k, const void* v, void* o, int B
 
 int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale,
                              int causal, int scan_order, int dtype, void* stream, const attn_fwd_opts* opts) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
-    if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device index %d is beyond the %d this entry point keeps track of", dev, kMaxDevices);
-    if (!g_noalloc_ptr[dev]) {
-        // Set-up, once per device, with that device current.  In host code the array's name is only a handle for
-        // this lookup, not an address a kernel could use; the lookup gives the address inside the current device.
-        int* ptr = nullptr;
-        e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch);
-        if (e != cudaSuccess || !ptr) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e)); }
-        g_noalloc_ptr[dev] = ptr;
-    }
+    // The first call on a device looks the scratch array's address up there (see current_device); later calls reuse it.
+    DeviceState ds;
+    int rc = current_device(&ds, nullptr);
+    if (rc) return rc;
     // fwd_common turns a launch of more than ATTN_NOALLOC_MAX_CTAS CTAs away before anything is enqueued.
-    return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, g_noalloc_ptr[dev], sizeof(g_noalloc_scratch),
+    return fwd_common(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, stream, opts, ds.noalloc_scratch, sizeof(g_noalloc_scratch),
                       ATTN_NOALLOC_MAX_CTAS);
 }
 
-static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
-                      int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, int* work_counter, size_t counter_bytes,
-                      int counter_ctas_max) {
+// Everything that can be refused is refused here, before anything is enqueued.
+struct Checked {
+    Resolved r;
+    DeviceState ds;
+    int dev;
+};
+static int check_call(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                      int scan_order, int dtype, const attn_fwd_opts* opts, bool dynamic, Checked* c) {
     if (!q || !k || !v || !o) return fail(ATTN_ERR_INVALID_ARG, "q, k, v and o must be non-null");
     int rc = check_shape(B, H, N, d, causal, dtype);
     if (rc) return rc;
     if (scan_order != ATTN_SCAN_CYCLIC && scan_order != ATTN_SCAN_SAWTOOTH)
         return fail(ATTN_ERR_INVALID_ARG, "unknown scan_order %d", scan_order);
-    if (!std::isfinite(scale) || !(scale > 0.f)) return fail(ATTN_ERR_INVALID_ARG, "scale must be finite and positive");
+    if (!std::isfinite(scale)) return fail(ATTN_ERR_INVALID_ARG, "scale must be finite");
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u)
         return fail(ATTN_ERR_ALIGNMENT, "q, k, v and o must be 16-byte aligned");
-    int sm_count = 0, smem_limit = 0;
-    rc = device_sm_count(&sm_count, &smem_limit);
+    if (opts && opts->lse && ((uintptr_t)opts->lse & 3u)) return fail(ATTN_ERR_ALIGNMENT, "opts->lse must be 4-byte aligned");
+    rc = current_device(&c->ds, &c->dev);
     if (rc) return rc;
-    Resolved r;
-    rc = resolve_opts(opts, d, smem_limit, &r);
+    return resolve_opts(opts, d, causal, dynamic, c->ds.smem_optin, &c->r);
+}
+
+static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
+                      int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, int* work_counter, size_t counter_bytes,
+                      int counter_ctas_max) {
+    Checked c;
+    int rc = check_call(q, k, v, o, B, H, N, d, scale, causal, scan_order, dtype, opts, work_counter != nullptr, &c);
     if (rc) return rc;
+    const Resolved& r = c.r;
 
     KernelParams kp;
     // Dynamic schedule: items are claimed in index order, and under the causal mask that order runs from the last
     // (longest) Q block of a head to the first, so that the short items fill the end of the launch.
     kp.sched = make_sched(B, H, N, r.q_tiles, r.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH, r.head_fastest,
-                          work_counter != nullptr && causal);
+                          work_counter != nullptr && causal, r.pairing);
     kp.work_counter = work_counter;
-    kp.scale_log2 = scale * 1.4426950408889634f;
+    // softmax(scale * s) is computed as 2^(|scale| log2(e) * (+-s) - m).  A scale of exactly zero (every visible key gets
+    // the same weight) runs as the smallest positive scale: the products then vanish against m, masked keys keep -inf.
+    const float mag = scale == 0.f ? 1e-30f : std::fabs(scale);
+    kp.scale_log2 = mag * 1.4426950408889634f;
+    kp.negate = scale < 0.f;
     kp.kv_stages = r.stages;
     kp.l2_policy = r.l2_policy;
     kp.o = o;
-    rc = (int)cudaGetSymbolAddress((void**)&kp.status, g_status_word);
-    if (rc != 0) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress failed (%d)", rc); }
-    rc = (int)cudaGetSymbolAddress((void**)&kp.cycles, g_cycles);
-    if (rc != 0) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaGetSymbolAddress failed (%d)", rc); }
+    kp.lse = opts ? opts->lse : nullptr;
+    kp.status = c.ds.status;
+    kp.cycles = c.ds.cycles;
 
-    CUtensorMap tq, tk, tv;
-    if ((rc = make_map(&tq, q, B * H, N, d, kBlockM, dtype))) return rc;
-    if ((rc = make_map(&tk, k, B * H, N, d, r.block_n, dtype))) return rc;
-    if ((rc = make_map(&tv, v, B * H, N, d, r.block_n, dtype))) return rc;
-    // O is written through shared memory, each softmax warp storing boxes of its d/2 columns x as many rows (at most its
-    // 32) as its eighth of a ring slot holds.
-    CUtensorMap to;
-    const int stage_row_bytes = d, stage_bytes_per_warp = r.block_n * d * 2 / 8;
-    const int stage_rows = stage_bytes_per_warp / stage_row_bytes < 32 ? stage_bytes_per_warp / stage_row_bytes : 32;
-    if ((rc = make_map(&to, o, B * H, N, d, stage_rows, dtype, d / 2))) return rc;
+    MapKey key;
+    key.q = q; key.k = k; key.v = v; key.o = o;
+    key.BH = B * H; key.N = N; key.d = d; key.dtype = dtype; key.block_n = r.block_n;
+    key.stage_rows = (r.block_n * d * 2 / 2 / 4) / 128 < 32 ? (r.block_n * d * 2 / 2 / 4) / 128 : 32;
+    const MapSet* maps = nullptr;
+    if ((rc = maps_for(key, &maps))) return rc;
 
-    const int grid = grid_for(kp.sched.n_work, sm_count, r);
+    const int grid = grid_for(kp.sched.n_units, c.ds.sm_count, r);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (work_counter) {
         if (r.launch_mode != 0) return fail(ATTN_ERR_INVALID_ARG, "the dynamic schedule needs the persistent launch (launch_mode 0)");
@@ -354,8 +463,11 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
         cudaError_t e = cudaMemsetAsync(work_counter, 0, (size_t)ATTN_DYNAMIC_SCRATCH_HEADER + 4u * (size_t)grid, st);
         if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "clearing the scratch: %s", cudaGetErrorString(e)); }
     }
-    return d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, tq, tk, tv, to, kp, grid, r.smem, st)
-                    : launch_tiles<64>(r.block_n, r.q_tiles, dtype, tq, tk, tv, to, kp, grid, r.smem, st);
+    rc = d == 128 ? launch_tiles<128>(r.block_n, r.q_tiles, dtype, c.dev, c.ds, *maps, kp, grid, r.smem, st)
+                  : launch_tiles<64>(r.block_n, r.q_tiles, dtype, c.dev, c.ds, *maps, kp, grid, r.smem, st);
+    if (rc) return rc;
+    // check_mode: wait for the device and report a wait that ran out inside the kernel as this call's status.
+    return r.check_mode ? read_status(nullptr) : ATTN_OK;
 }
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
@@ -364,35 +476,32 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H,
 }
 
 namespace {
-// Streams and events of the attn_fwd_host pipeline, one set per device, created on first use.
+// Streams and events of the attn_fwd_host pipeline, one set per device, created on first use.  One call at a time
+// enqueues on a device's set: the set's mutex is held from the first event record to the last.
 struct HostPipe {
+    std::mutex busy;
     bool ready = false;
     cudaStream_t up = nullptr, run = nullptr, down = nullptr;
-    cudaEvent_t start = nullptr, done = nullptr, uploaded[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {};
+    cudaEvent_t start = nullptr, done_up = nullptr, done_run = nullptr, done_down = nullptr;
+    cudaEvent_t uploaded[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {};
 };
 HostPipe g_host_pipe[kMaxDevices];
-std::mutex g_host_pipe_mutex;
 
-int host_pipe_for_current_device(HostPipe** out) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e)); }
-    if (dev < 0 || dev >= kMaxDevices) return fail(ATTN_ERR_UNSUPPORTED, "device index %d is beyond the %d the host pipeline keeps track of", dev, kMaxDevices);
-    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
-    HostPipe& hp = g_host_pipe[dev];
-    if (!hp.ready) {
-        bool ok = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&hp.run, cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
-        for (int i = 0; ok && i < kMaxHostChunks; ++i)
-            ok = cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
-        if (!ok) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "creating the streams and events of the host pipeline failed"); }
-        hp.ready = true;
-    }
-    *out = &hp;
+// Called with hp.busy held.
+int prepare_host_pipe(HostPipe& hp) {
+    if (hp.ready) return ATTN_OK;
+    bool ok = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.run, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done_up, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done_run, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done_down, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kMaxHostChunks; ++i)
+        ok = cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "creating the streams and events of the host pipeline failed"); }
+    hp.ready = true;
     return ATTN_OK;
 }
 }  // namespace
@@ -401,15 +510,20 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
                   void* v_dev, void* o_dev, int B, int H, int N, int d, float scale, int causal, int scan_order, int dtype,
                   void* stream, const attn_fwd_opts* opts) {
     if (!q_host || !k_host || !v_host || !o_host) return fail(ATTN_ERR_INVALID_ARG, "host buffers must be non-null");
-    if (!q_dev || !k_dev || !v_dev || !o_dev) return fail(ATTN_ERR_INVALID_ARG, "device staging buffers must be non-null");
-    int rc = check_shape(B, H, N, d, causal, dtype);
+    // Every argument and option is checked before the first copy is enqueued.
+    Checked c;
+    int rc = check_call(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, opts, false, &c);
     if (rc) return rc;
+    if (c.r.check_mode) return fail(ATTN_ERR_INVALID_ARG, "check_mode would make attn_fwd_host wait inside its pipeline: call attn_device_status afterwards instead");
+    attn_fwd_opts inner;
+    memset(&inner, 0, sizeof(inner));
+    if (opts) inner = *opts;
+    inner.lse = nullptr;   // the groups of heads below are separate launches with their own [heads, N] numbering
     const size_t bytes = (size_t)B * H * N * d * 2;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e;
+    cudaError_t e = cudaSuccess;
     const long long heads = (long long)B * H;
-    int chunks = opts ? opts->host_chunks : 0;
-    if (chunks < 0 || chunks > kMaxHostChunks) return fail(ATTN_ERR_INVALID_ARG, "host_chunks must be in [0, %d]", kMaxHostChunks);
+    int chunks = inner.host_chunks;
     if (chunks == 0) chunks = bytes > ((size_t)32 << 20) ? 8 : 1;
     if (chunks > heads) chunks = (int)heads;
     if (chunks <= 1) {
@@ -419,7 +533,7 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
             cudaGetLastError();
             return fail(ATTN_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
         }
-        rc = attn_fwd_ex(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, stream, opts);
+        rc = attn_fwd_ex(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, stream, &inner);
         if (rc) return rc;
         if ((e = cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) {
             cudaGetLastError();
@@ -428,36 +542,50 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
         return ATTN_OK;
     }
     // Pipeline over groups of heads: upload, kernel and download of successive groups overlap on three streams.
-    HostPipe* hp = nullptr;
-    if ((rc = host_pipe_for_current_device(&hp))) return rc;
+    HostPipe& hp = g_host_pipe[c.dev];
+    std::lock_guard<std::mutex> lock(hp.busy);
+    if ((rc = prepare_host_pipe(hp))) return rc;
     const size_t head_bytes = (size_t)N * d * 2;
-    auto fail_cuda = [&](const char* what) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e)); };
-    if ((e = cudaEventRecord(hp->start, st)) != cudaSuccess) return fail_cuda("cudaEventRecord");
-    if ((e = cudaStreamWaitEvent(hp->up, hp->start, 0)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->run, hp->start, 0)) != cudaSuccess ||
-        (e = cudaStreamWaitEvent(hp->down, hp->start, 0)) != cudaSuccess)
-        return fail_cuda("cudaStreamWaitEvent");
+    const char* what = "";
+    if ((e = cudaEventRecord(hp.start, st)) != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaEventRecord: %s", cudaGetErrorString(e)); }
+    // From here on the side streams may hold work: whatever happens, `stream` is made to wait for all three before returning.
+    bool failed = false;
+    auto check = [&](cudaError_t err, const char* where) {
+        if (err != cudaSuccess && !failed) { failed = true; e = err; what = where; cudaGetLastError(); }
+        return err == cudaSuccess;
+    };
+    check(cudaStreamWaitEvent(hp.up, hp.start, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(hp.run, hp.start, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(hp.down, hp.start, 0), "cudaStreamWaitEvent");
     long long h0 = 0;
-    for (int c = 0; c < chunks; ++c) {
-        const long long n_heads = heads / chunks + (c < heads % chunks ? 1 : 0);
+    for (int ch = 0; ch < chunks && !failed && rc == 0; ++ch) {
+        const long long n_heads = heads / chunks + (ch < heads % chunks ? 1 : 0);
         const size_t off = (size_t)h0 * head_bytes, len = (size_t)n_heads * head_bytes;
         const uint8_t *qh = (const uint8_t*)q_host + off, *kh = (const uint8_t*)k_host + off, *vh = (const uint8_t*)v_host + off;
         uint8_t *qd = (uint8_t*)q_dev + off, *kd = (uint8_t*)k_dev + off, *vd = (uint8_t*)v_dev + off, *od = (uint8_t*)o_dev + off;
-        if ((e = cudaMemcpyAsync(qd, qh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess ||
-            (e = cudaMemcpyAsync(kd, kh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess ||
-            (e = cudaMemcpyAsync(vd, vh, len, cudaMemcpyHostToDevice, hp->up)) != cudaSuccess)
-            return fail_cuda("host-to-device copy");
-        if ((e = cudaEventRecord(hp->uploaded[c], hp->up)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->run, hp->uploaded[c], 0)) != cudaSuccess)
-            return fail_cuda("cudaEventRecord");
-        rc = attn_fwd_ex(qd, kd, vd, od, 1, (int)n_heads, N, d, scale, causal, scan_order, dtype, hp->run, opts);
-        if (rc) return rc;
-        if ((e = cudaEventRecord(hp->computed[c], hp->run)) != cudaSuccess || (e = cudaStreamWaitEvent(hp->down, hp->computed[c], 0)) != cudaSuccess)
-            return fail_cuda("cudaEventRecord");
-        if ((e = cudaMemcpyAsync((uint8_t*)o_host + off, od, len, cudaMemcpyDeviceToHost, hp->down)) != cudaSuccess)
-            return fail_cuda("device-to-host copy");
+        if (!check(cudaMemcpyAsync(qd, qh, len, cudaMemcpyHostToDevice, hp.up), "host-to-device copy") ||
+            !check(cudaMemcpyAsync(kd, kh, len, cudaMemcpyHostToDevice, hp.up), "host-to-device copy") ||
+            !check(cudaMemcpyAsync(vd, vh, len, cudaMemcpyHostToDevice, hp.up), "host-to-device copy") ||
+            !check(cudaEventRecord(hp.uploaded[ch], hp.up), "cudaEventRecord") ||
+            !check(cudaStreamWaitEvent(hp.run, hp.uploaded[ch], 0), "cudaStreamWaitEvent"))
+            break;
+        rc = attn_fwd_ex(qd, kd, vd, od, 1, (int)n_heads, N, d, scale, causal, scan_order, dtype, hp.run, &inner);
+        if (rc) break;
+        if (!check(cudaEventRecord(hp.computed[ch], hp.run), "cudaEventRecord") ||
+            !check(cudaStreamWaitEvent(hp.down, hp.computed[ch], 0), "cudaStreamWaitEvent") ||
+            !check(cudaMemcpyAsync((uint8_t*)o_host + off, od, len, cudaMemcpyDeviceToHost, hp.down), "device-to-host copy"))
+            break;
         h0 += n_heads;
     }
-    if ((e = cudaEventRecord(hp->done, hp->down)) != cudaSuccess || (e = cudaStreamWaitEvent(st, hp->done, 0)) != cudaSuccess)
-        return fail_cuda("cudaEventRecord");
+    // Join: `stream` continues only after everything enqueued on the three side streams, on success and on failure alike.
+    check(cudaEventRecord(hp.done_up, hp.up), "cudaEventRecord");
+    check(cudaEventRecord(hp.done_run, hp.run), "cudaEventRecord");
+    check(cudaEventRecord(hp.done_down, hp.down), "cudaEventRecord");
+    check(cudaStreamWaitEvent(st, hp.done_up, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(st, hp.done_run, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(st, hp.done_down, 0), "cudaStreamWaitEvent");
+    if (rc) return rc;   // attn_fwd_ex's own message stands
+    if (failed) return fail(ATTN_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
     return ATTN_OK;
 }
 
@@ -480,19 +608,6 @@ int attn_debug_profile(unsigned long long* out) {
 }
 #endif
 
-int attn_device_status(int* code) {
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e)); }
-    int word = 0;
-    e = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int));
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(ATTN_ERR_CUDA, "reading the status word: %s", cudaGetErrorString(e)); }
-    if (code) *code = word;
-    if (word != 0) {
-        const int zero = 0;
-        cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int));
-        return fail(ATTN_ERR_DEVICE_TIMEOUT, "kernel wait site %d ran out of time", word);
-    }
-    return ATTN_OK;
-}
+int attn_device_status(int* code) { return read_status(code); }
 
 }  // extern "C"

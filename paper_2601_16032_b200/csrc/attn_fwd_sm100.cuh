@@ -2,19 +2,11 @@
 // S, P and O in tensor memory, one softmax thread per query row, O written by TMA stores.
 //
 // One CTA handles work items of kQTiles x 128 query rows (Algorithm 1's resident Q tile).  Warp roles:
-//   eight softmax warps    two threads per query row: warps w and w + 4 own TMEM lanes 32 (w % 4) .. + 31,
-//                          the first the lower half of a tile's key columns (and of O's columns), the
-//                          second the upper half.  All eight work on the SAME Q tile at a time and take
-//                          the tiles of a work item in turn, K/V step by K/V step: while they run the
-//                          softmax of one tile the tensor core runs the other tile's products, and one
-//                          tile's softmax has the whole SM's exponential throughput and issue slots, which
-//                          halves the latency between a tile's S and its P.  A thread reads its half of S
-//                          from TMEM, swaps its partial row maximum with its partner through shared memory
-//                          (an mbarrier per warp pair), keeps the running max and a partial sum, writes P
-//                          back over its own S columns as 16-bit pairs in two parts, rescales its half of
-//                          O when the max moved, and at the end of the item normalises its half of the O
-//                          row and stages it in shared memory, from where one lane per warp issues a TMA
-//                          store.
+//   the softmax warps      one warpgroup per Q tile, thread r owning row r (TMEM lane r).  A thread reads its
+//                          row of S from TMEM, keeps the running max and sum, writes P back to TMEM as 16-bit
+//                          pairs in two parts, rescales its row of O when the max moved, and at the end of the
+//                          item normalises the O row and stages it in shared memory, from where one lane per
+//                          warp issues a TMA store.
 //   the next warp          producer: one elected lane issues the TMA loads (Q tiles, then K_j, V_j in
 //                          the scan order of the item, then one empty slot: the item's O staging buffer)
 //                          into a ring of shared-memory slots.
@@ -22,6 +14,7 @@
 //                          O_q += P_q V_j and commits them to mbarriers; the first of them also owns
 //                          the TMEM allocation.
 //   the remaining warp(s)  idle; they complete the warpgroup whose registers go to the softmax threads.
+// With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
 // Work items come from Algorithm 2's grid-stride walk or, with a counter in global memory, are claimed
 // dynamically; Algorithm 4's scan direction follows the CTA's own item count either way.
 #pragma once
@@ -45,10 +38,12 @@ __device__ unsigned long long g_profile[256][32];
 
 struct KernelParams {
     SchedParams sched;
-    float scale_log2;     // scale * log2(e): probabilities are computed with ex2
+    float scale_log2;     // |scale| * log2(e): probabilities are computed with ex2
+    int negate;           // 1: scale < 0, the scores change sign before anything else is done with them
     int kv_stages;        // slots in the K/V ring
     int l2_policy;        // 1: K/V loads evict_last, Q loads evict_first
     void* o;              // [B, H, N, d] output
+    float* lse;           // [B, H, N] natural-log sum of exponentials per query row, or nullptr
     int* status;          // device status word (0 = fine)
     unsigned long long* cycles;  // CTA 0 leaves the SM cycles its MMA loop took here
     int* work_counter;    // dynamic schedule: [0] next unclaimed work index (zero at launch), [64 + cta] items the CTA
@@ -66,7 +61,7 @@ constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the
 enum WaitSite {
     kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
     kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8, kSiteWorkFull = 9, kSiteWorkEmpty = 10,
-    kSiteStageSlot = 11, kSiteStageDone = 12, kSiteExchange = 13
+    kSiteStageSlot = 11, kSiteStageDone = 12
 };
 
 struct __align__(8) Barriers {
@@ -74,14 +69,11 @@ struct __align__(8) Barriers {
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
     uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
     uint64_t drain[2];
-    uint64_t stage_done;                    // staged epilogue: the eight softmax warps have read their staging buffers out
-    uint64_t pair[4];                       // per pair of softmax warps (w, w + 4): both have published their partial row value
+    uint64_t stage_done[2];                 // staged epilogue: the four warps of Q tile q have read their staging buffers out
     uint64_t work_full[2], work_empty[2];  // dynamic schedule: two-slot mailbox of claimed work indices
     long long work_k[2];
     uint32_t tmem_base;
     int abort_flag;
-    float xchg[2][2][128];  // [exchange count & 1][column half][row]: the partial row maximum (or, at the end of an item,
-                            // the partial row sum) each thread of a row shows its partner
 };
 
 template <int kD, int kBlockN, int kQTiles>
@@ -91,30 +83,29 @@ struct Geometry {
     static constexpr int kKVTileBytes = kBlockN * kD * 2;
     static constexpr int kQChunkBytes = kBlockM * 128;
     static constexpr int kKVChunkBytes = kBlockN * 128;
-    static constexpr int kColsS = kBlockN / 2;              // S columns a softmax thread owns (two threads per row)
-    static constexpr int kColsO = kD / 2;                   // O columns a softmax thread owns
+    static constexpr int kColsS = kBlockN;                  // S columns a softmax thread owns: its whole row
+    static constexpr int kColsO = kD;                       // O columns a softmax thread owns
+    // Epilogue through shared memory: after the last V tile of a work item the ring holds one more slot that
+    // nothing is loaded into; the softmax warps of Q tile q stage their 16-bit O rows in half q of it, kStageRows rows
+    // of one 64-column block per warp at a time, and write them out with TMA stores (full 128-byte lines, rows
+    // beyond N dropped by the copy engine).
+    static constexpr int kStageBytesPerWarp = kKVTileBytes / 2 / 4;
+    static constexpr int kStageRows = kStageBytesPerWarp / 128 < 32 ? kStageBytesPerWarp / 128 : 32;
     // P reaches the MMA warp in two parts: a thread announces its first kEarlyGroups groups of 16
-    // probabilities (one K step of the P.V product each) while it still computes the rest.  A thread writes its
-    // P over the first half of its own S columns, so the 16 keys of K step kk of the P.V product sit at column
-    // (kk / kGroups) * kColsS + (kk % kGroups) * 8 of the tile's S block.
+    // probabilities (one K step of the P.V product each) while it still computes the rest.
     static constexpr int kGroups = kColsS / 16;
     static constexpr int kEarlyGroups = kGroups >= 4 ? (kGroups * 3) / 4 : kGroups / 2;
-    static constexpr int kSoftmaxWarps = 8;
-    static constexpr int kSoftmaxThreads = kSoftmaxWarps * 32;
-    static constexpr int kThreads = kSoftmaxThreads + 128;  // plus one warpgroup: producer, MMA warps, idle warp(s)
-    // Epilogue through shared memory: after the last V tile of a work item the ring holds one more slot that
-    // nothing is loaded into.  Each softmax warp owns an eighth of it and stages there, one Q tile after the other,
-    // kStageRows rows of its kColsO 16-bit O columns at a time, written out by TMA stores (rows beyond N are
-    // dropped by the copy engine).
-    static constexpr int kStageBytesPerWarp = kKVTileBytes / kSoftmaxWarps;
-    static constexpr int kStageRowBytes = kColsO * 2;       // 128 (d = 128) or 64 (d = 64)
-    static constexpr int kStageRows = kStageBytesPerWarp / kStageRowBytes < 32 ? kStageBytesPerWarp / kStageRowBytes : 32;
-    // Registers: the launch gives each of the 384 threads 65536 / 384 rounded down to a multiple of 8 = 168; the last
-    // warpgroup hands registers back and the softmax warpgroups take them (256 * 200 + 128 * 104 = 384 * 168).
+    static constexpr int kSoftmaxWarps = kQTiles * 4;
+    static constexpr int kTileThreads = 128;                // softmax threads of one Q tile
+    static constexpr int kThreads = kSoftmaxWarps * 32 + 128;  // plus one warpgroup: producer, MMA warps, idle warp(s)
+    // Registers: the launch gives every thread 65536 / kThreads rounded down to a multiple of 8.  With two Q tiles
+    // that is 168 (384 threads): the last warpgroup hands registers back and the softmax warpgroups take them
+    // (256 * 200 + 128 * 104 = 384 * 168).
+    static constexpr bool kRebalance = (kQTiles == 2);
     static constexpr int kRegsOther = 104;
     static constexpr int kRegsSoftmax = 200;
     static constexpr int kTmemCols = 512;
-    static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q overwrites parts of it
+    static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q aliases its first kBlockN/2 columns
     static constexpr int kTmemO = 256;    // O_q (fp32, kD columns) at kTmemO + 128 q
     static constexpr size_t smem_bytes(int stages) {
         return (size_t)kQTiles * kQTileBytes + (size_t)stages * kKVTileBytes + sizeof(Barriers);
@@ -174,16 +165,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         for (int q = 0; q < 2; ++q) {
             ptx::mbar_init(&bar->s_full[q], 1);
-            ptx::mbar_init(&bar->p_early[q], G::kSoftmaxWarps);
-            ptx::mbar_init(&bar->p_full[q], G::kSoftmaxWarps);
+            ptx::mbar_init(&bar->p_early[q], 4);   // one arrival per softmax warp of the tile
+            ptx::mbar_init(&bar->p_full[q], 4);
             ptx::mbar_init(&bar->o_full[q], 1);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&bar->work_full[i], 1);
             ptx::mbar_init(&bar->work_empty[i], kQTiles + G::kSoftmaxWarps);
         }
-        for (int i = 0; i < 4; ++i) ptx::mbar_init(&bar->pair[i], 2);
-        ptx::mbar_init(&bar->stage_done, G::kSoftmaxWarps);
+        ptx::mbar_init(&bar->stage_done[0], 4);
+        ptx::mbar_init(&bar->stage_done[1], 4);
         ptx::mbar_init(&bar->drain[0], 1);
         ptx::mbar_init(&bar->drain[1], 1);
         bar->abort_flag = 0;
@@ -204,17 +195,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     ptx::tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
 
-    // Which work item this CTA handles as its iteration `it` (-1: none left).  Static schedule (Algorithm 2):
-    // blockIdx.x + it * gridDim.x.  Dynamic schedule: the producer warp claims the next unclaimed index from a
-    // global counter and passes it to the other roles through a two-slot mailbox in shared memory, so a CTA
-    // that drew short items simply draws more of them; Algorithm 4's parity stays the CTA's own count `it`.
+    // Which work item this CTA handles as its item number `it`.  Static schedule (Algorithm 2): the CTA walks the
+    // units blockIdx.x, += gridDim.x; `slot` counts the positions of that walk (a unit holds one or two items).
+    // Dynamic schedule: the producer warp claims the next unclaimed item from a global counter and passes it to the
+    // other roles through a two-slot mailbox in shared memory, so a CTA that drew short items simply draws more of
+    // them.  Algorithm 4's parity is the CTA's own count `it` either way.
     const bool dynamic = p.work_counter != nullptr;
-    auto static_work = [&](int it) -> long long {
-        const long long k = (long long)blockIdx.x + (long long)it * gridDim.x;
-        return k < p.sched.n_work ? k : -1;
+    auto static_next = [&](int& slot, int it, WorkItem& w) -> bool {
+        for (;;) {
+            const Slot sl = static_slot(p.sched, (int)blockIdx.x, (int)gridDim.x, slot++);
+            if (sl.kind == kSlotEnd) return false;
+            if (sl.kind == kSlotItem) { w = make_item(p.sched, sl.bh, sl.q_item, it); return true; }
+        }
     };
-    auto claim_work = [&](int it, bool& ok) -> long long {  // producer warp, all lanes
-        if (!dynamic) return static_work(it);
+    auto claimed_item = [&](long long claim, int it) -> WorkItem {
+        const Slot sl = claimed_slot(p.sched, claim);
+        return make_item(p.sched, sl.bh, sl.q_item, it);
+    };
+    auto claim_work = [&](int it, bool& ok) -> long long {  // producer warp, all lanes (dynamic schedule)
         const int slot = it & 1;
         if (it >= 2) {
             ok = ptx::warp_all(ptx::mbar_wait(&bar->work_empty[slot], (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag, kSiteWorkEmpty));
@@ -228,8 +226,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         __syncwarp();
         return bar->work_k[slot];
     };
-    auto take_work = [&](int it, bool& ok, bool whole_warp) -> long long {  // MMA lanes (one thread), softmax warps
-        if (!dynamic) return static_work(it);
+    auto take_work = [&](int it, bool& ok, bool whole_warp) -> long long {  // MMA lanes (one thread), softmax warps (dynamic schedule)
         const int slot = it & 1;
         if (!ptx::mbar_wait(&bar->work_full[slot], (uint32_t)((it >> 1) & 1), abort_flag, kSiteWorkFull)) { ok = false; return -1; }
         const long long k = bar->work_k[slot];
@@ -245,7 +242,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (warp >= G::kSoftmaxWarps) {
     // The last warpgroup (producer, MMA and idle warps) hands registers back in one instruction.  (Its three
     // roles below keep the indentation of the outer level.)
-    ptx::reg_dealloc<G::kRegsOther>();
+    if (G::kRebalance) ptx::reg_dealloc<G::kRegsOther>();
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
         // The whole warp walks the schedule and waits on the barriers; one elected lane issues the
@@ -256,11 +253,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t q_issued = 0;     // Q loads issued so far
         long long kv_issued = 0;   // K/V tile loads issued so far
         bool ok = true;
-        int it = 0;
+        int it = 0, slot = 0;
         for (; ok; ++it) {
-            const long long k = claim_work(it, ok);
-            if (!ok || k < 0) break;
-            const WorkItem w = decode_work(p.sched, k, it);
+            WorkItem w;
+            if (dynamic) {
+                const long long k = claim_work(it, ok);
+                if (!ok || k < 0) break;
+                w = claimed_item(k, it);
+            } else if (!static_next(slot, it, w)) {
+                break;
+            }
             ok = ptx::warp_all(ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ));
             if (!ok) break;
             if (ptx::elect_one()) {
@@ -360,8 +362,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk) {
                 if (((kk % G::kGroups) >= G::kEarlyGroups) != (late != 0)) continue;
-                ptx::mma_ts(o_tmem, s_tmem + (kk / G::kGroups) * G::kColsS + (kk % G::kGroups) * 8,
-                            b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv, accumulate | (late != 0) | (kk != 0));
+                ptx::mma_ts(o_tmem, s_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
+                            accumulate | (late != 0) | (kk != 0));
             }
         };
 
@@ -370,11 +372,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (ptx::elect_one()) {
             const long long clk_begin = clock64();
             SAW_PROF_DECL;
-            int it = 0;
+            int it = 0, slot = 0;
             for (; ok; ++it) {
-                const long long k = take_work(it, ok, false);
-                if (!ok || k < 0) break;
-                const WorkItem w = decode_work(p.sched, k, it);
+                WorkItem w;
+                if (dynamic) {
+                    const long long k = take_work(it, ok, false);
+                    if (!ok || k < 0) break;
+                    w = claimed_item(k, it);
+                } else if (!static_next(slot, it, w)) {
+                    break;
+                }
                 const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
                 SAW_PROF(0);
                 if (!ptx::mbar_wait(&bar->q_full, it & 1, abort_flag, kSiteMmaQ)) { ok = false; break; }
@@ -433,8 +440,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (!ok) break;
                 if (hi_mine > 0) ptx::mma_commit(&bar->o_full[q]);
-                // The staging slot is released by the softmax warps on behalf of every tile they stored, and here for a
-                // tile that lies beyond N.
+                // The staging slot is released by the tile's softmax warps, or here if the tile lies beyond N.
                 if (hi_mine == 0) ptx::mbar_arrive(&bar->kv_empty[ring.slot]);
                 ring.advance(stages);
             }
@@ -448,276 +454,229 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     } else {
         // ------------------------------------------------------------------ softmax / correction / epilogue
-        ptx::reg_alloc<G::kRegsSoftmax>();
+        if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
         constexpr int kColsS = G::kColsS, kColsO = G::kColsO;
-        const int half = warp >> 2;                    // which half of a row's key columns and of its O columns
-        const int wq = warp & 3;                       // which quarter of the tile's rows = of the TMEM lanes
-        const int r_in_tile = wq * 32 + lane;          // row inside a tile = TMEM lane
-        const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
-        const uint32_t t_s0 = tmem + lane_base + G::kTmemS + half * kColsS;   // + 128 q: this thread's S (and P) columns
-        const uint32_t t_o0 = tmem + lane_base + G::kTmemO + half * kColsO;   // + 128 q: this thread's O columns
-        uint64_t* pair_bar = &bar->pair[wq];
+        const int q = warp >> 2;                       // which Q tile this thread works on
+        const int r_in_tile = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + G::kTmemS + 128 * q;
+        const uint32_t t_p = t_s;                      // P overwrites the first half of the row's S columns
+        const uint32_t t_o = tmem + lane_base + G::kTmemO + 128 * q;
         const float scale_log2 = p.scale_log2;
         const int N = p.sched.N;
-        uint32_t s_phases = 0, o_phases = 0;   // bit q: parity of the next phase of s_full[q] / o_full[q]
-        uint32_t xcount = 0;       // exchanges with the partner thread so far (picks the buffer and the barrier phase)
+        uint32_t s_phase = 0, o_phase = 0;
         bool ok = true;
-        int it = 0;
+        int it = 0, slot = 0;
         Ring ring;                 // position of the next work item's first K tile in the K/V ring
         uint32_t stage_phase = 0;
         SAW_PROF_DECL;
-        // The two threads of a row show each other a partial value (row maximum, row sum) through shared memory: show()
-        // publishes this thread's, partner() waits for the other's.  Successive exchanges alternate between two buffers.
-        auto show = [&](float mine) {
-            bar->xchg[xcount & 1][half][r_in_tile] = mine;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(pair_bar);
-        };
-        auto partner = [&](float& theirs) -> bool {
-            const bool got = ptx::mbar_wait(pair_bar, xcount & 1u, abort_flag, kSiteExchange);
-            theirs = bar->xchg[xcount & 1][half ^ 1][r_in_tile];
-            ++xcount;
-            return got;
-        };
         for (; ok; ++it) {
-            const long long k = take_work(it, ok, true);
-            if (!ok || k < 0) break;
-            const WorkItem w = decode_work(p.sched, k, it);
+            WorkItem w;
+            if (dynamic) {
+                const long long k = take_work(it, ok, true);
+                if (!ok || k < 0) break;
+                w = claimed_item(k, it);
+            } else if (!static_next(slot, it, w)) {
+                break;
+            }
+            const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
             ring.advance_by(2 * w.hi, stages);   // now at the item's staging slot
             const Ring stage = ring;
             ring.advance(stages);
-            // Running max (the reference the exponents are taken against, log2 units) and this thread's partial sum
-            // of probabilities, for the tile handled now (_a) and for the other one (_b).
-            float m_a = -INFINITY, l_a = 0.f, m_b = -INFINITY, l_b = 0.f;
-            bool first_a = true, first_b = true;
-            for (int s = 0; ok && s < w.hi; ++s) {
+            if (hi_mine == 0) continue;
+            const int tile_row0 = w.row0 + q * kBlockM;
+            const int row = tile_row0 + r_in_tile;
+            float m_ref = -INFINITY;   // the max the exponents are taken against (log2 units)
+            float l = 0.f;             // running sum of this thread's probabilities
+            bool first = true;
+            for (int s = 0; s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
+                if (j >= hi_mine) continue;
+                SAW_PROF(0);
+                const bool got_s = ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS);
+                s_phase ^= 1u;
+                ptx::tc_fence_after();
+                SAW_PROF(1);
+
+                uint32_t sv[kColsS / 32][32];
+#pragma unroll
+                for (int c = 0; c < kColsS / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
+                ptx::tmem_wait_ld();
+                SAW_PROF(2);
+
+                if (p.negate) {   // a negative scale: work on -S with |scale|
+#pragma unroll
+                    for (int c = 0; c < kColsS / 32; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) sv[c][i] ^= 0x80000000u;
+                }
+                const int col0 = j * kBlockN;  // key index of the row's first column
+                const bool masked = (j * kBlockN + kBlockN > N) || (p.sched.causal && (j * kBlockN + kBlockN - 1 > tile_row0));
+                if (masked) {
+                    const int limit = p.sched.causal ? (row < N - 1 ? row : N - 1) : N - 1;  // last visible key
+#pragma unroll
+                    for (int c = 0; c < kColsS / 32; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + c * 32 + i > limit) sv[c][i] = 0xff800000u;  // -inf
+                }
+
+                // Eight independent chains of three-input maxima, then a tree.
+                float mx[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mx[i] = ptx::max3(__uint_as_float(sv[0][3 * i]), __uint_as_float(sv[0][3 * i + 1]), __uint_as_float(sv[0][3 * i + 2]));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mx[i] = ptx::max3(mx[i], __uint_as_float(sv[0][24 + 2 * i]), __uint_as_float(sv[0][25 + 2 * i]));
+#pragma unroll
+                for (int c = 1; c < kColsS / 32; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2)
+                        mx[(i >> 1) & 7] = ptx::max3(mx[(i >> 1) & 7], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
+                float row_max = fmaxf(ptx::max3(mx[0], mx[1], mx[2]), fmaxf(ptx::max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                SAW_PROF(3);
+                ok = ptx::warp_all(got_s);
+                if (!ok) break;
+                SAW_PROF(4);
+                const float m_cand = fmaxf(m_ref, row_max * scale_log2);
+                const bool need = (m_cand - m_ref) > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    float alpha = 1.f;
+                    if (need) {
+                        alpha = ptx::ex2(m_ref - m_cand);  // 0 when nothing was accumulated yet
+                        m_ref = m_cand;
+                        l *= alpha;
+                    }
+                    if (!first) {
+                        // S_q is complete, so every product issued before it, O_q's last update included, is too.
 #pragma unroll 1
-                for (int q = 0; q < kQTiles; ++q) {
-                    const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
-                    if (j < hi_mine) {
-                        const int tile_row0 = w.row0 + q * kBlockM;
-                        const int row = tile_row0 + r_in_tile;
-                        const uint32_t t_s = t_s0 + 128 * q, t_o = t_o0 + 128 * q;
-                        SAW_PROF(0);
-                        const bool got_s = ptx::mbar_wait(&bar->s_full[q], (s_phases >> q) & 1u, abort_flag, kSiteSoftmaxS);
-                        s_phases ^= 1u << q;
-                        ptx::tc_fence_after();
-                        SAW_PROF(1);
-
-                        uint32_t sv[kColsS / 32][32];
+                        for (int c = 0; c < kColsO / 16; ++c) {
+                            uint32_t ov[16];
+                            ptx::tmem_ld16(t_o + c * 16, ov);
+                            ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < kColsS / 32; ++c) ptx::tmem_ld32(t_s + c * 32, sv[c]);
-                        ptx::tmem_wait_ld();
-                        SAW_PROF(2);
-
-                        const int col0 = j * kBlockN + half * kColsS;  // key index of this thread's first column
-                        const bool masked = (j * kBlockN + kBlockN > N) || (p.sched.causal && (j * kBlockN + kBlockN - 1 > tile_row0));
-                        if (masked) {
-                            const int limit = p.sched.causal ? (row < N - 1 ? row : N - 1) : N - 1;  // last visible key
-#pragma unroll
-                            for (int c = 0; c < kColsS / 32; ++c)
-#pragma unroll
-                                for (int i = 0; i < 32; ++i)
-                                    if (col0 + c * 32 + i > limit) sv[c][i] = 0xff800000u;  // -inf
+                            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                            ptx::tmem_st16(t_o + c * 16, ov);
                         }
-
-                        // Eight independent chains of three-input maxima, then a tree.
-                        float mx[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) mx[i] = ptx::max3(__uint_as_float(sv[0][3 * i]), __uint_as_float(sv[0][3 * i + 1]), __uint_as_float(sv[0][3 * i + 2]));
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) mx[i] = ptx::max3(mx[i], __uint_as_float(sv[0][24 + 2 * i]), __uint_as_float(sv[0][25 + 2 * i]));
-#pragma unroll
-                        for (int c = 1; c < kColsS / 32; ++c)
-#pragma unroll
-                            for (int i = 0; i < 32; i += 2)
-                                mx[(i >> 1) & 7] = ptx::max3(mx[(i >> 1) & 7], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
-                        float row_max = fmaxf(ptx::max3(mx[0], mx[1], mx[2]), fmaxf(ptx::max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                        // The two threads of a row swap their maxima.  (Both have loaded their S columns by now and each
-                        // writes P over its own columns only, so neither can overwrite what the other still has to read.)
-                        show(row_max);
-                        const ptx::f32x2 scale2 = ptx::pack_f32x2(scale_log2, scale_log2);
-                        ptx::f32x2 l01 = ptx::pack_f32x2(0.f, 0.f), l23 = ptx::pack_f32x2(0.f, 0.f);
-                        // Groups of 16 probabilities (eight packed registers, one TMEM store each): x = S * scale * log2(e) - m
-                        // as packed FMAs, then 2^x on the MUFU or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
-                        uint32_t pk[G::kGroups][8];
-                        auto exp_group = [&](int g, ptx::f32x2 neg_m2) {
-                            const int c = g >> 1, h = g & 1;
-#pragma unroll
-                            for (int i = 0; i < 16; i += 4) {
-                                const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
-                                const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
-                                float x0, x1, x2, x3, p0, p1, p2, p3;
-                                ptx::unpack_f32x2(xa, x0, x1);
-                                ptx::unpack_f32x2(xb, x2, x3);
-                                if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
-                                else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
-                                if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
-                                else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
-                                l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
-                                l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
-                                pk[g][i / 2] = ptx::pack2<kBf16>(p0, p1);
-                                pk[g][i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
-                            }
-                        };
-                        // While the partner's maximum is on its way the first group is computed against the reference the
-                        // row already has: the reference moves only when the row maximum grew by more than the threshold,
-                        // which is rare after an item's first steps.  When it does move, the group is computed again.
-                        float neg_m = (m_a == -INFINITY) ? 0.f : -m_a;
-                        ptx::f32x2 neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
-                        exp_group(0, neg_m2);
-                        SAW_PROF(3);
-                        float other_max;
-                        const bool got_x = partner(other_max);
-                        ok = ptx::warp_all(got_s && got_x);
-                        if (!ok) break;
-                        row_max = fmaxf(row_max, other_max);
-                        SAW_PROF(4);
-                        const float m_cand = fmaxf(m_a, row_max * scale_log2);
-                        const bool need = (m_cand - m_a) > kRescaleThreshold;
-                        if (__any_sync(0xffffffffu, need)) {
-                            float alpha = 1.f;
-                            if (need) {
-                                alpha = ptx::ex2(m_a - m_cand);  // 0 when nothing was accumulated yet
-                                m_a = m_cand;
-                                l_a *= alpha;
-                            }
-                            if (!first_a) {
-                                // S_q is complete, so every product issued before it, O_q's last update included, is too.
-#pragma unroll 1
-                                for (int c = 0; c < kColsO / 16; ++c) {
-                                    uint32_t ov[16];
-                                    ptx::tmem_ld16(t_o + c * 16, ov);
-                                    ptx::tmem_wait_ld();
-#pragma unroll
-                                    for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                                    ptx::tmem_st16(t_o + c * 16, ov);
-                                }
-                            }
-                            neg_m = (m_a == -INFINITY) ? 0.f : -m_a;
-                            neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
-                            l01 = ptx::pack_f32x2(0.f, 0.f);
-                            l23 = ptx::pack_f32x2(0.f, 0.f);
-                            exp_group(0, neg_m2);
-                        }
-                        SAW_PROF(5);
-                        // The store of a group is issued after the exponentials of the next group, so that it never waits
-                        // in the instruction stream for MUFU results that are still in flight.
-                        auto finish_group = [&](int g) {
-                            ptx::tmem_st8(t_s + g * 8, pk[g]);
-                            if (g == G::kEarlyGroups - 1) {
-                                ptx::tmem_wait_st();
-                                ptx::tc_fence_before();
-                                __syncwarp();
-                                if (lane == 0) ptx::mbar_arrive(&bar->p_early[q]);
-                                SAW_PROF(6);
-                            }
-                        };
-#pragma unroll
-                        for (int g = 1; g < G::kGroups; ++g) {
-                            exp_group(g, neg_m2);
-                            finish_group(g - 1);
-                        }
-                        finish_group(G::kGroups - 1);
-                        float l0, l1, l2, l3;
-                        ptx::unpack_f32x2(l01, l0, l1);
-                        ptx::unpack_f32x2(l23, l2, l3);
-                        l_a += (l0 + l1) + (l2 + l3);
+                    }
+                }
+                SAW_PROF(5);
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                const ptx::f32x2 scale2 = ptx::pack_f32x2(scale_log2, scale_log2);
+                const ptx::f32x2 neg_m2 = ptx::pack_f32x2(neg_m, neg_m);
+                ptx::f32x2 l01 = ptx::pack_f32x2(0.f, 0.f), l23 = ptx::pack_f32x2(0.f, 0.f);
+                // Groups of 16 probabilities (eight packed registers, one TMEM store each).  The store of a
+                // group is issued after the exponentials of the next group, so that it never waits in the
+                // instruction stream for MUFU results that are still in flight.
+                uint32_t pk[G::kGroups][8];
+                auto finish_group = [&](int g) {
+                    ptx::tmem_st8(t_p + g * 8, pk[g]);
+                    if (g == G::kEarlyGroups - 1) {
                         ptx::tmem_wait_st();
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bar->p_full[q]);
-                        SAW_PROF(7);
-                        first_a = false;
+                        if (lane == 0) ptx::mbar_arrive(&bar->p_early[q]);
+                        SAW_PROF(6);
                     }
-                    if (kQTiles == 2) {   // the other tile's state takes its turn
-                        const float tm = m_a, tl = l_a;
-                        const bool tf = first_a;
-                        m_a = m_b; l_a = l_b; first_a = first_b;
-                        m_b = tm; l_b = tl; first_b = tf;
+                };
+#pragma unroll
+                for (int g = 0; g < G::kGroups; ++g) {
+                    const int c = g >> 1, h = g & 1;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        // Four probabilities: x = S * scale * log2(e) - m as two packed FMAs, then 2^x on the MUFU
+                        // or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
+                        const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
+                        const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
+                        float x0, x1, x2, x3, p0, p1, p2, p3;
+                        ptx::unpack_f32x2(xa, x0, x1);
+                        ptx::unpack_f32x2(xb, x2, x3);
+                        if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
+                        else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
+                        if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
+                        else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
+                        l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
+                        l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
+                        pk[g][i / 2] = ptx::pack2<kBf16>(p0, p1);
+                        pk[g][i / 2 + 1] = ptx::pack2<kBf16>(p2, p3);
                     }
+                    if (g > 0) finish_group(g - 1);
                 }
+                finish_group(G::kGroups - 1);
+                float l0, l1, l2, l3;
+                ptx::unpack_f32x2(l01, l0, l1);
+                ptx::unpack_f32x2(l23, l2, l3);
+                l += (l0 + l1) + (l2 + l3);
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bar->p_full[q]);
+                SAW_PROF(7);
+                first = false;
             }
             if (!ok) break;
-            // ---- epilogue, one Q tile after the other: O_q / l -> 16 bit -> staging rows -> TMA store
-            int tiles_stored = 0;
-#pragma unroll 1
-            for (int q = 0; q < kQTiles; ++q) {
-                const int hi_mine = q ? w.hi_q[1] : w.hi_q[0];
-                if (hi_mine > 0) {
-                    const int tile_row0 = w.row0 + q * kBlockM;
-                    const uint32_t t_o = t_o0 + 128 * q;
-                    SAW_PROF(0);
-                    const bool got_o = ptx::mbar_wait(&bar->o_full[q], (o_phases >> q) & 1u, abort_flag, kSiteSoftmaxO);
-                    o_phases ^= 1u << q;
-                    ptx::tc_fence_after();
-                    SAW_PROF(9);
-                    float other_sum;
-                    show(l_a);
-                    const bool got_x = partner(other_sum);
-                    const bool got_slot = ptx::mbar_wait(&bar->kv_full[stage.slot], stage.phase, abort_flag, kSiteStageSlot);
-                    ok = ptx::warp_all(got_o && got_x && got_slot);
-                    if (!ok) break;
-                    SAW_PROF(10);
-                    const float inv_l = 1.f / (l_a + other_sum);
-                    uint8_t* buf = kv_smem + (size_t)stage.slot * G::kKVTileBytes + (size_t)warp * G::kStageBytesPerWarp;
-                    const int my_pass = lane / G::kStageRows, my_row = lane % G::kStageRows;
-                    uint32_t pk[kColsO / 2];   // this thread's O columns of the row, 16-bit pairs
+            // ---- epilogue: O_q / l -> 16 bit -> global
+            SAW_PROF(0);
+            const bool got_o = ptx::mbar_wait(&bar->o_full[q], o_phase, abort_flag, kSiteSoftmaxO);
+            o_phase ^= 1u;
+            ptx::tc_fence_after();
+            SAW_PROF(9);
+            ok = ptx::warp_all(got_o);
+            if (!ok) break;
+            const float inv_l = 1.f / l;
+            // ln sum_j exp(scale * s_j) of the row: the probabilities were taken as 2^(x - m_ref), so the sum is 2^m_ref * l.
+            if (p.lse != nullptr && row < N) p.lse[(size_t)w.bh * N + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
+            ok = ptx::warp_all(ptx::mbar_wait(&bar->kv_full[stage.slot], stage.phase, abort_flag, kSiteStageSlot));
+            if (!ok) break;
+            SAW_PROF(10);
+            uint8_t* buf = kv_smem + (size_t)stage.slot * G::kKVTileBytes + (size_t)q * (G::kKVTileBytes / 2) +
+                           (size_t)(warp & 3) * G::kStageBytesPerWarp;
+            const int my_pass = lane / G::kStageRows, my_row = lane % G::kStageRows;
 #pragma unroll
-                    for (int c = 0; c < kColsO / 32; ++c) {
-                        uint32_t ov[32];
-                        ptx::tmem_ld32(t_o + c * 32, ov);
-                        ptx::tmem_wait_ld();
+            for (int c64 = 0; c64 < kD / 64; ++c64) {
+                uint32_t pk[32];   // this row's 64 columns of the block, 16-bit pairs
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2)
-                            pk[c * 16 + i / 2] = ptx::pack2<kBf16>(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l);
-                    }
-#pragma unroll 1
-                    for (int ps = 0; ps < 32 / G::kStageRows; ++ps) {
-                        if (my_pass == ps) {
-                            // Rows of 128 (64) bytes, eight to a 1024 (512)-byte swizzle atom: 16-byte piece i of row r sits
-                            // at piece i ^ (r & 7) (i ^ ((r >> 1) & 3)).
-                            uint4* dst_row = reinterpret_cast<uint4*>(buf + my_row * G::kStageRowBytes);
-                            const int sw = G::kStageRowBytes == 128 ? (my_row & 7) : ((my_row >> 1) & 3);
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t ov[32];
+                    ptx::tmem_ld32(t_o + c64 * 64 + hf * 32, ov);
+                    ptx::tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < G::kStageRowBytes / 16; ++i)
-                                dst_row[i ^ sw] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-                        }
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        const int y0 = tile_row0 + wq * 32 + ps * G::kStageRows;
-                        if (y0 < N && ptx::elect_one()) {   // rows of the box beyond N are dropped by the copy
-                            ptx::tma_store_3d(&tm_o, buf, half * kColsO, y0, w.bh);
-                            ptx::bulk_commit_group();
-                            ptx::bulk_wait_group_read0();   // the buffer may be written again
-                        }
-                        __syncwarp();
-                    }
-                    ++tiles_stored;
-                    ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
-                    SAW_PROF(11);
+                    for (int i = 0; i < 32; i += 2)
+                        pk[hf * 16 + i / 2] = ptx::pack2<kBf16>(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l);
                 }
-                if (kQTiles == 2) {
-                    const float tm = m_a, tl = l_a;
-                    m_a = m_b; l_a = l_b;
-                    m_b = tm; l_b = tl;
+#pragma unroll 1
+                for (int ps = 0; ps < 32 / G::kStageRows; ++ps) {
+                    if (my_pass == ps) {
+                        // 128-byte rows, eight to a 1024-byte swizzle atom: 16-byte piece i of row r sits at piece i ^ (r & 7)
+                        uint4* dst_row = reinterpret_cast<uint4*>(buf + my_row * 128);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst_row[i ^ (my_row & 7)] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    const int y0 = tile_row0 + (warp & 3) * 32 + ps * G::kStageRows;
+                    if (y0 < N && ptx::elect_one()) {   // rows of the box beyond N are dropped by the copy
+                        ptx::tma_store_3d(&tm_o, buf, c64 * 64, y0, w.bh);
+                        ptx::bulk_commit_group();
+                        ptx::bulk_wait_group_read0();   // the buffer may be written again
+                    }
+                    __syncwarp();
                 }
             }
-            if (!ok) break;
-            // The slot goes back to the producer once all eight warps have read their buffers out: one arrival per tile
-            // stored (the MMA lane of a tile beyond N makes that tile's).
-            if (lane == 0) ptx::mbar_arrive(&bar->stage_done);
-            if (warp == 0) {
-                ok = ptx::warp_all(ptx::mbar_wait(&bar->stage_done, stage_phase, abort_flag, kSiteStageDone));
-                if (ok && lane == 0)
-                    for (int t = 0; t < tiles_stored; ++t) ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
+            SAW_PROF(11);
+            // The slot goes back to the producer once the four warps of the tile have read their buffers out.
+            if (lane == 0) ptx::mbar_arrive(&bar->stage_done[q]);
+            if ((warp & 3) == 0) {
+                ok = ptx::warp_all(ptx::mbar_wait(&bar->stage_done[q], stage_phase, abort_flag, kSiteStageDone));
+                if (ok && lane == 0) ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
             }
             stage_phase ^= 1u;
+            if (!ok) break;
+            ptx::tc_fence_before();  // ordered before this thread's next arrive on p_full, which lets O_q be overwritten
             SAW_PROF(8);
         }
         ptx::bulk_wait_group0();   // this thread's TMA stores have landed before the CTA ends
-        SAW_PROF_WRITE(12, warp == 0 && lane == 0);
+        SAW_PROF_WRITE(12, q == 0 && r_in_tile == 0);
     }
 
     ptx::tc_fence_before();

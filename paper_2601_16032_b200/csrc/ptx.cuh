@@ -33,24 +33,6 @@ __device__ __forceinline__ bool elect_one() {
 }
 __device__ __forceinline__ bool warp_all(bool x) { return __all_sync(0xffffffffu, x) != 0; }
 
-// Named barriers over `count` threads of the CTA (ids 1..15; 0 is __syncthreads).  The reducing form
-// returns the AND of every participant's flag, the same value in all of them.
-__device__ __forceinline__ void bar_sync(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-__device__ __forceinline__ bool bar_red_and(int id, int count, bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %3, 0;\n\t"
-        "bar.red.and.pred q, %1, %2, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r)
-        : "r"(id), "r"(count), "r"((uint32_t)flag)
-        : "memory");
-    return r != 0;
-}
-
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -1,6 +1,6 @@
 """Per-phase SM-cycle breakdown of the attention kernel, from in-kernel clock stamps.
 
-    python -m paper_2601_16032_b200.profile_phases [B H N d] [--causal] [--fp16]
+    python profile_phases.py [B H N d] [--causal] [--fp16] [--cyclic]
 
 Builds a second copy of the library with -DSAW_PROFILE (libsawtooth_attn_profile.so, beside the normal one), runs one
 warmed-up launch of the given shape (default 4 16 8192 128, bf16, non-causal, sawtooth order) and prints, for the
@@ -14,14 +14,20 @@ import ctypes
 import os
 import subprocess
 
+import sys
+
 import numpy as np
 
-from . import build as _build
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_16032_b200 import build as _build
 
 PROFILE_LIB = os.path.join(_build.PKG, "libsawtooth_attn_profile.so")
 MMA_PHASES = ["loop / decode", "wait Q", "wait K/V", "wait P (early part)", "issue P.V (early)", "wait P (rest)", "issue P.V (rest)",
               "issue Q.K + commit", "release K/V slots"]
-SOFTMAX_PHASES = ["loop / decode", "wait S", "TMEM load", "mask + row max", "max exchange", "rescale test", "exp, convert, store (early part)",
+SOFTMAX_PHASES = ["loop / decode", "wait S", "TMEM load", "mask + row max", "warp vote", "rescale test", "exp, convert, store (early part)",
                   "exp, convert, store (rest) + arrive", "epilogue: rest", "epilogue: wait O", "epilogue: wait staging slot",
                   "epilogue: stage + TMA store"]
 
@@ -77,10 +83,17 @@ def main() -> None:
     cycles = ctypes.c_ulonglong(0)
     lib.attn_last_kernel_cycles(ctypes.byref(cycles))
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    items = B * H * -(-N // 256)
-    grid = min(items, sms)
-    a = np.frombuffer(table, dtype=np.uint64).reshape(256, 32)[:grid].astype(np.float64)
-    steps = -(-items // grid) * (-(-N // 128)) / (2.0 if args.causal else 1.0)  # K/V steps of the busiest CTA (about, if causal)
+    # K/V steps per CTA from the host replay of the schedule (the normal library's; the schedule is the same).
+    import paper_2601_16032_b200 as sa
+    trace = sa.attn_schedule_trace(B, H, N, d, int(args.causal), sa.CYCLIC if args.cyclic else sa.SAWTOOTH,
+                                   sa.F16 if args.fp16 else sa.BF16, None, sms)
+    per_cta = {}
+    for e in trace:
+        per_cta[e.cta] = per_cta.get(e.cta, 0) + e.n_kv
+    grid = len(per_cta)
+    a = np.frombuffer(table, dtype=np.uint64).reshape(256, 32)[:min(grid, 256)].astype(np.float64)
+    steps = float(np.median([per_cta[c] for c in range(min(grid, 256))]))  # K/V steps of the median CTA
+    cycles.value = int(cycles.value * steps / per_cta[0])                  # CTA 0's cycle count, scaled to that many steps
     ms = e0.elapsed_time(e1)
     flops = 4.0 * B * H * float(N) ** 2 * d / (2 if args.causal else 1)
     print(f"B={B} H={H} N={N} d={d} {'fp16' if args.fp16 else 'bf16'} {'causal' if args.causal else 'non-causal'} "

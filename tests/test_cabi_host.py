@@ -95,16 +95,39 @@ SHAPES = [
 @pytest.mark.parametrize("order", [sa.CYCLIC, sa.SAWTOOTH])
 @pytest.mark.parametrize("digits", [sa.TILE_FASTEST, sa.HEAD_FASTEST])
 def test_schedule_replay_equals_the_schedule_oracle(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits):
+    check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits, sa.PAIR_NONE, "none")
+
+
+@pytest.mark.parametrize("n_sm,B,H,N,d,q_tiles,block_n", SHAPES + [(5, 1, 3, 2305, 128, 2, 128)])
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("order", [sa.CYCLIC, sa.SAWTOOTH])
+@pytest.mark.parametrize("pairing", [(sa.PAIR_MIRRORED, "mirrored"), (sa.PAIR_ADJACENT, "adjacent")])
+def test_paired_schedule_replay_equals_the_schedule_oracle(n_sm, B, H, N, d, q_tiles, block_n, causal, order, pairing):
+    check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, sa.TILE_FASTEST, pairing[0], pairing[1])
+    check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, sa.HEAD_FASTEST, pairing[0], pairing[1])
+
+
+def test_default_pairing_is_mirrored_under_the_causal_mask_only():
+    assert sa.attn_query_plan(1, 32, 32768, 128, 1, sa.BF16, sm_count=148).pairing == sa.PAIR_MIRRORED
+    assert sa.attn_query_plan(1, 32, 32768, 128, 0, sa.BF16, sm_count=148).pairing == sa.PAIR_NONE
+    p = sa.attn_query_plan(1, 32, 32768, 128, 1, sa.BF16, sm_count=148)
+    assert p.n_units == 32 * 64 and p.grid == 148
     o = sa.Opts()
-    o.q_tiles, o.block_n, o.digit_order = q_tiles, block_n, digits
+    o.pairing = sa.PAIR_NONE
+    assert sa.attn_query_plan(1, 32, 32768, 128, 1, sa.BF16, o, sm_count=148).n_units == 32 * 128
+
+
+def check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits, pairing, pairing_name):
+    o = sa.Opts()
+    o.q_tiles, o.block_n, o.digit_order, o.pairing = q_tiles, block_n, digits, pairing
     got = sa.attn_schedule_trace(B, H, N, d, causal, order, sa.F16, o, sm_count=n_sm)
     W = 128 * q_tiles
     want = [w for seq in sch.full_schedule(n_sm, B, H, N, W, block_n, bool(causal), order,
-                                           "head_fastest" if digits else "tile_fastest") for w in seq]
+                                           "head_fastest" if digits else "tile_fastest", pairing=pairing_name) for w in seq]
     assert len(got) == len(want)
     for g, w in zip(got, want):
-        assert (g.cta, g.iteration, g.k, g.batch, g.head, g.q_item, bool(g.backward), g.n_kv) == \
-            (w.cta, w.i_local, w.k, w.batch, w.head, w.q_tile, w.backward, w.n_kv)
+        assert (g.cta, g.iteration, g.k, g.batch, g.head, g.q_item, bool(g.backward), g.n_kv, g.member) == \
+            (w.cta, w.i_local, w.k, w.batch, w.head, w.q_tile, w.backward, w.n_kv, w.member)
         # per 128-row tile ranges: what an item of W = 128 rows at that position would need
         for qi, n_q in enumerate((g.n_kv_q0, g.n_kv_q1)):
             r = g.q_item * W + qi * 128

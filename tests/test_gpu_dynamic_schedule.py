@@ -15,6 +15,8 @@ def run_dynamic(w, qkv, order, opts=None, ctas_for_scratch=None):
     import paper_2601_16032_b200 as sa
     q, k, v = qkv
     adt = sa.BF16 if w.dtype == wl.BF16 else sa.F16
+    opts = opts or sa.Opts()
+    opts.pairing = sa.PAIR_NONE   # the dynamic schedule claims single items: the plan that sizes its scratch has no pairs
     plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt, opts)
     n_bytes = sa.attn_dynamic_scratch_bytes(plan.grid if ctas_for_scratch is None else ctas_for_scratch)
     scratch = torch.full((n_bytes // 4,), 0x5a5a5a5a, dtype=torch.int32, device=q.device)  # stale contents on purpose
@@ -83,3 +85,7 @@ def test_dynamic_rejects_bad_scratch_and_launch_mode():
     opts.launch_mode = 1
     with pytest.raises(sa.AttnError):
         run_dynamic(w, qkv, sa.CYCLIC, opts)
+    opts = sa.Opts()
+    opts.pairing = sa.PAIR_MIRRORED
+    with pytest.raises(sa.AttnError):
+        sa.attn_fwd_dynamic(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), 1, 2, 512, 64, 0.125, 1, 0, sa.F16, 0, opts, q.data_ptr(), 4096)

@@ -49,7 +49,8 @@ def test_tile_shapes_and_scan_orders(block_n, q_tiles, causal, d, dtype):
 
 
 @pytest.mark.parametrize("opt", [dict(kv_stages=2), dict(kv_stages=3), dict(digit_order=1), dict(launch_mode=1),
-                                 dict(l2_policy=1), dict(max_ctas=1)])
+                                 dict(l2_policy=1), dict(max_ctas=1), dict(pairing=1), dict(pairing=2), dict(pairing=3),
+                                 dict(pairing=2, launch_mode=1), dict(pairing=3, digit_order=1, max_ctas=2), dict(check_mode=1)])
 def test_options_do_not_change_the_result(opt):
     import paper_2601_16032_b200 as sa
     w = wl.small_workload("opts", 2, 2, 900, 128, wl.BF16, True, 7200)
@@ -128,7 +129,7 @@ def test_bad_arguments_are_rejected_before_launch():
     p = t.data_ptr()
     st = 0
     cases = [
-        (dict(q=0), -1), (dict(N=0), -1), (dict(d=96), -2), (dict(scale=float("nan")), -1), (dict(scale=-1.0), -1),
+        (dict(q=0), -1), (dict(N=0), -1), (dict(d=96), -2), (dict(scale=float("nan")), -1), (dict(scale=float("inf")), -1),
         (dict(scan_order=5), -1), (dict(dtype=7), -1), (dict(causal=2), -1), (dict(q=p + 2), -3),
     ]
     for change, status in cases:
@@ -197,3 +198,98 @@ def test_monotonically_growing_scores_and_uniform_scores():
             sa.attn_device_status()
             err = np.abs(o[0, 0].double().cpu().numpy() - want)
             assert err.max() <= 2e-2 and err.mean() <= 2e-3, (causal, order, err.max(), err.mean())
+
+
+@pytest.mark.parametrize("pairing", [1, 2, 3])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("N,q_tiles", [(2305, 2), (1330, 1), (256, 2), (300, 2)])
+def test_pairings_cover_every_row(pairing, causal, N, q_tiles):
+    """One item per unit, mirrored pairs and adjacent pairs (odd and even numbers of Q blocks, a head of one block),
+    few CTAs so that every CTA walks several units: every row of every head against the oracle, both scan orders."""
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("pairs", 1, 3, N, 128, wl.BF16, causal, 7400 + N)
+    qkv = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        assert_parity(w, run_cuda(w, qkv, order, opts_for(q_tiles=q_tiles, pairing=pairing, max_ctas=2)))
+
+
+@pytest.mark.parametrize("scale", [-0.11, 0.0, -2.5])
+@pytest.mark.parametrize("causal", [False, True])
+def test_negative_and_zero_scale(scale, causal):
+    """Any finite scale: a negative one turns the softmax towards the smallest scores, zero weighs every visible key
+    alike (O is the mean, or prefix mean, of V).  Against the oracle, which takes the scale as it is."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    from oracle import attention as ora
+    w = wl.small_workload("scale", 1, 2, 900, 64, wl.F16, causal, 7450)
+    q, k, v = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        o = sa.forward(q, k, v, causal=causal, scan_order=order, scale=scale)
+        sa.attn_device_status()
+        for h in range(w.H):
+            want = ora.attention_head(*(wl.bits_to_f64(wl.head_bits(w, n, 0, h), w.dtype) for n in ("q", "k", "v")), scale, causal)
+            err = np.abs(o[0, h].double().cpu().numpy() - want)
+            assert err.max() <= 2e-2 and err.mean() <= 2e-3, (scale, causal, order, err.max(), err.mean())
+
+
+def test_host_entry_point_refuses_before_copying_and_leaves_the_stream_usable():
+    """A bad option makes attn_fwd_host fail before anything is enqueued (the device staging buffers keep their
+    contents); a good call on the same stream afterwards gives the device entry point's result bit for bit."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("host-bad", 1, 5, 700, 128, wl.BF16, True, 7351)
+    q, k, v = upload(w)
+    want = run_cuda(w, (q, k, v), sa.CYCLIC)
+    host = [t.view(torch.int16).cpu().pin_memory() for t in (q, k, v)]
+    o_host = torch.full(q.shape, -1, dtype=torch.int16).pin_memory()
+    dev = [torch.full_like(q.view(torch.int16), 77) for _ in range(4)]
+    stream = torch.cuda.Stream()
+
+    def call(opts, scan_order=sa.CYCLIC):
+        sa.attn_fwd_host(host[0].data_ptr(), host[1].data_ptr(), host[2].data_ptr(), o_host.data_ptr(), dev[0].data_ptr(),
+                         dev[1].data_ptr(), dev[2].data_ptr(), dev[3].data_ptr(), w.B, w.H, w.N, w.d, w.scale, 1, scan_order,
+                         sa.BF16, stream.cuda_stream, opts)
+
+    for bad in (dict(block_n=96), dict(kv_stages=99), dict(pairing=9), dict(check_mode=1)):
+        opts = sa.Opts()
+        opts.host_chunks = 3
+        for name, val in bad.items():
+            setattr(opts, name, val)
+        with pytest.raises(sa.AttnError):
+            call(opts)
+    opts = sa.Opts()
+    opts.host_chunks = 3
+    with pytest.raises(sa.AttnError):
+        call(opts, scan_order=7)
+    stream.synchronize()
+    assert all((d == 77).all() for d in dev)        # nothing was copied
+    call(opts)
+    stream.synchronize()
+    sa.attn_device_status()
+    assert torch.equal(o_host, want.view(torch.int16).cpu())
+
+
+def test_repeated_calls_reuse_cached_tensor_maps_correctly():
+    """The library keeps the tensor maps of the last few (pointers, shape) combinations a thread used: alternating between
+    two sets of buffers, and reusing one buffer with another shape, must keep giving each call its own result."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    wa = wl.small_workload("maps-a", 1, 2, 640, 128, wl.BF16, False, 7500)
+    wb = wl.small_workload("maps-b", 1, 2, 640, 128, wl.BF16, False, 7501)
+    a, b = upload(wa), upload(wb)
+    want_a, want_b = run_cuda(wa, a, sa.CYCLIC), run_cuda(wb, b, sa.CYCLIC)
+    for _ in range(3):
+        assert torch.equal(run_cuda(wa, a, sa.CYCLIC), want_a)
+        assert torch.equal(run_cuda(wb, b, sa.CYCLIC), want_b)
+    # same buffers read as one head of twice the length
+    wc = wl.small_workload("maps-c", 1, 1, 1280, 128, wl.BF16, True, 7502)
+    qc, kc, vc = (t.view(1, 1, 1280, 128) for t in a)
+    o = torch.empty_like(qc)
+    sa.attn_fwd(qc.data_ptr(), kc.data_ptr(), vc.data_ptr(), o.data_ptr(), 1, 1, 1280, 128, wc.scale, 1, sa.CYCLIC, sa.BF16,
+                torch.cuda.current_stream().cuda_stream)
+    sa.attn_device_status()
+    from oracle import attention as ora
+    f = lambda t: t[0, 0].double().cpu().numpy()
+    err = np.abs(f(o) - ora.attention_head(f(qc), f(kc), f(vc), wc.scale, True))
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    assert torch.equal(run_cuda(wa, a, sa.CYCLIC), want_a)

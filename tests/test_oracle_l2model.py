@@ -73,3 +73,43 @@ def test_wavefront_trace_of_a_schedule():
     assert l2model.lru_misses(tr, 2) == 4 + 2
     s = sch.full_schedule(2, 1, 1, 512, 128, 128, False, sch.CYCLIC)
     assert l2model.lru_misses(l2model.wavefront_trace(s), 2) == 8
+
+
+def causal_misses(n_sm, H, N, capacity_tiles, order, pairing):
+    s = sch.full_schedule(n_sm, 1, H, N, 256, 128, True, order, pairing=pairing)
+    return l2model.lru_misses(l2model.wavefront_trace(s), capacity_tiles)
+
+
+@pytest.mark.parametrize("heads_in_cache", [0.5, 2])
+def test_lru_on_causal_schedules_unpaired_sawtooth_loses_and_mirrored_pairs_win(heads_in_cache):
+    """A scaled-down causal workload (16 CTAs, 8 heads of 64 K/V tiles, 256-row items) through an ideal LRU cache.
+    Without pairs the items of a wave differ in length, the CTAs drift apart, and backward scans that start at each
+    item's own diagonal make it worse: the sawtooth order misses more than the cyclic one.  With mirrored pairs every
+    unit is equally long, the wave stays on a few tiles, and the sawtooth order is never the worse one."""
+    n_sm, H, N = 16, 8, 8192
+    cap = int(heads_in_cache * N // 128)
+    compulsory = H * N // 128
+    none_cyc = causal_misses(n_sm, H, N, cap, sch.CYCLIC, "none")
+    none_saw = causal_misses(n_sm, H, N, cap, sch.SAWTOOTH, "none")
+    mir_cyc = causal_misses(n_sm, H, N, cap, sch.CYCLIC, "mirrored")
+    mir_saw = causal_misses(n_sm, H, N, cap, sch.SAWTOOTH, "mirrored")
+    assert none_saw > none_cyc > 4 * compulsory
+    assert compulsory <= mir_saw <= mir_cyc <= 2 * compulsory
+    assert mir_saw * 4 < none_cyc
+
+
+def test_mirrored_sawtooth_wave_reads_two_tiles_at_a_time():
+    """One head, W = B_c, CTAs in lockstep: a CTA on pair p reads tile t at step t < n-p (first member, forward) and tile
+    n - t afterwards (second member, backward), whatever p is, so the whole wave touches at most two tiles per step."""
+    N, W, n_sm = 4096, 128, 8
+    n = N // W
+    s = sch.full_schedule(n_sm, 1, 1, N, W, W, True, sch.SAWTOOTH, pairing="mirrored")
+    per_cta = [[j for w in seq[:2] for j in w.kv_order()] for seq in s]     # every CTA's first unit
+    assert all(len(steps) == n + 1 for steps in per_cta)
+    for t in range(n + 1):
+        tiles = {steps[t] for steps in per_cta}
+        assert tiles <= {t, n - t}
+    # the cyclic order spreads the second members over as many tiles as there are CTAs
+    c = sch.full_schedule(n_sm, 1, 1, N, W, W, True, sch.CYCLIC, pairing="mirrored")
+    per_cta = [[j for w in seq[:2] for j in w.kv_order()] for seq in c]
+    assert len({steps[n - 1] for steps in per_cta}) == n_sm

@@ -179,3 +179,50 @@ def test_rejects_bad_arguments():
         ora.attention_rows(q, np.array([0, 9]), rnd((3, 4), 2), rnd((3, 4), 3), 1.0, False)
     with pytest.raises(ValueError):
         ora.attention_rows(q, np.array([0, 1]), rnd((3, 5), 2), rnd((3, 4), 3), 1.0, False)
+
+
+@pytest.mark.parametrize("n,_,d", CASES)
+@pytest.mark.parametrize("causal", [False, True])
+def test_logsumexp_matches_scipy(n, _, d, causal):
+    """Library routine: scipy's logsumexp over the masked score rows."""
+    q, k = rnd((n, d), 21), rnd((n, d), 22)
+    scale = 0.41
+    s = scale * np.einsum("id,jd->ij", q, k)
+    if causal:
+        s[np.triu_indices(n, 1)] = -np.inf
+    want = scipy.special.logsumexp(s, axis=1)
+    rows = np.arange(n, dtype=np.int64)
+    np.testing.assert_allclose(ora.logsumexp_rows(q, rows, k, scale, causal), want, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(ora.logsumexp_definition(q, k, scale, causal), want, rtol=0, atol=1e-12)
+
+
+def test_logsumexp_closed_forms():
+    """K = 0 makes every score 0: the row sees c keys and lse = ln c (c = N, or i + 1 under the causal mask).  One
+    score far above the rest gives lse = that score.  Shifting every score of a row by a constant shifts lse by it."""
+    n, d = 37, 5
+    q, k0 = rnd((n, d), 23), np.zeros((n, d))
+    rows = np.arange(n, dtype=np.int64)
+    np.testing.assert_allclose(ora.logsumexp_rows(q, rows, k0, 0.7, False), np.full(n, np.log(n)), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(ora.logsumexp_rows(q, rows, k0, 0.7, True), np.log(rows + 1.0), rtol=0, atol=1e-13)
+    k = rnd((n, d), 24) * 0.01
+    k[11] = 50.0 * q[3] / np.dot(q[3], q[3])          # q[3] . k[11] = 50
+    got = ora.logsumexp_rows(q[3:4], np.array([3]), k, 2.0, False)
+    assert abs(got[0] - 100.0) < 1e-12
+    # appending a constant feature c to q and 1 to every k adds c to every score of the row
+    q1 = np.concatenate([q, np.full((n, 1), 3.25)], axis=1)
+    k1 = np.concatenate([k, np.ones((n, 1))], axis=1)
+    np.testing.assert_allclose(ora.logsumexp_rows(q1, rows, k1, 1.0, True) - ora.logsumexp_rows(q, rows, k, 1.0, True),
+                               np.full(n, 3.25), rtol=0, atol=1e-12)
+
+
+def test_logsumexp_normalises_the_definition():
+    """exp(s - lse) are the softmax weights: they sum to 1 and reproduce the attention output."""
+    n, d = 45, 9
+    q, k, v = rnd((n, d), 25), rnd((n, d), 26), rnd((n, d), 27)
+    scale = 0.5
+    lse = ora.logsumexp_rows(q, np.arange(n, dtype=np.int64), k, scale, True)
+    s = scale * (q @ k.T)
+    s[np.triu_indices(n, 1)] = -np.inf
+    w = np.exp(s - lse[:, None])
+    np.testing.assert_allclose(w.sum(axis=1), np.ones(n), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(w @ v, ora.attention_head(q, k, v, scale, True), rtol=0, atol=1e-13)

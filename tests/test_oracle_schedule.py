@@ -60,3 +60,43 @@ def test_max_ctas_limits_the_grid():
     s = sch.full_schedule(148, 1, 1, 4096, 128, 128, False, sch.SAWTOOTH, max_ctas=3)
     assert len(s) == 3
     assert [w.q_tile for w in s[1]] == list(range(1, 32, 3))
+
+
+@pytest.mark.parametrize("n_sm,B,H,N,W,B_c", SHAPES + [(3, 1, 2, 2305, 256, 128), (6, 2, 1, 4096, 256, 128)])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("order", [sch.CYCLIC, sch.SAWTOOTH])
+@pytest.mark.parametrize("pairing", ["mirrored", "adjacent"])
+def test_pairs_cover_every_q_tile_once_and_alternate(n_sm, B, H, N, W, B_c, causal, order, pairing):
+    s = sch.full_schedule(n_sm, B, H, N, W, B_c, causal, order, "tile_fastest", pairing=pairing)
+    n_q = sch.ceil_div(N, W)
+    n_units = B * H * sch.ceil_div(n_q, 2)
+    assert len(s) == min(n_units, n_sm)
+    seen = sorted((w.batch, w.head, w.q_tile) for seq in s for w in seq)
+    assert seen == sorted(itertools.product(range(B), range(H), range(n_q)))
+    for c, seq in enumerate(s):
+        assert sorted(set(w.k for w in seq)) == list(range(c, n_units, len(s)))   # units: k = blockIdx, += G
+        assert [w.i_local for w in seq] == list(range(len(seq)))
+        for w in seq:
+            assert w.backward == (order == sch.SAWTOOTH and w.i_local % 2 == 1)
+        for k, grp in itertools.groupby(seq, key=lambda w: w.k):
+            grp = list(grp)
+            assert [w.member for w in grp] == list(range(len(grp))) and 1 <= len(grp) <= 2
+            assert len({(w.batch, w.head) for w in grp}) == 1                     # both tiles of a pair in one head
+            p = k % sch.ceil_div(n_q, 2)
+            if pairing == "mirrored":
+                assert [w.q_tile for w in grp] == ([n_q - 1 - p, p] if n_q - 1 - p != p else [p])
+            else:
+                assert [w.q_tile for w in grp] == [t for t in (2 * p, 2 * p + 1) if t < n_q]
+
+
+def test_mirrored_pairs_are_equally_long_under_the_causal_mask():
+    """Tile t scans t+1 tiles' worth of K/V when W = B_c divides N, so the members of pair p scan (n-p) + (p+1) = n+1."""
+    N, W = 4096, 128
+    n_q = N // W
+    s = sch.full_schedule(5, 1, 3, N, W, W, True, sch.SAWTOOTH, pairing="mirrored")
+    for seq in s:
+        for _, grp in itertools.groupby(seq, key=lambda w: w.k):
+            assert sum(w.n_kv for w in grp) == n_q + 1
+    # without pairs the items of one CTA differ in length by up to the whole sequence
+    lengths = [w.n_kv for seq in sch.full_schedule(5, 1, 3, N, W, W, True, sch.SAWTOOTH) for w in seq]
+    assert min(lengths) == 1 and max(lengths) == n_q

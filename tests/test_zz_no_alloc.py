@@ -22,6 +22,7 @@ def test_no_alloc_entry_matches_the_scratch_taking_entry_twice_in_a_row():
     stream = torch.cuda.current_stream().cuda_stream
     opts = sa.Opts()
     opts.max_ctas = 5   # several items per CTA, so the counters are really used
+    opts.pairing = sa.PAIR_NONE   # the dynamic schedule claims single items
     plan = sa.attn_query_plan(w.B, w.H, w.N, w.d, 1, sa.BF16, opts)
     n_bytes = sa.attn_dynamic_scratch_bytes(plan.grid)
     scratch = torch.zeros(n_bytes // 4, dtype=torch.int32, device=q.device)
