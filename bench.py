@@ -48,10 +48,21 @@ FALLBACK_BF16_TFLOPS = 1590.0
 FLOP_PER_CLK_PER_SM = 8192.0
 WARMUP_LOAD_SECONDS = 0.25
 
-# DRAM bytes one launch moves (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture of the same kernel and
-# launch plan; the summaries under profiles/ name the captures).  Keyed by (workload, scan order); a workload that
-# has no capture of the present kernel reports null.
-NCU_DRAM_BYTES_PER_LAUNCH: dict = {}
+# DRAM bytes one launch moves: (dram__bytes_read.sum, dram__bytes_write.sum) of a one-launch ncu capture of the present
+# kernel on the full-size workload with the default launch plan (three metrics, one pass).
+# Keyed by (workload, scan order, pairing in force); anything else reports null.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("c3", "cyclic", "none"): (403114240, 116056576),
+    ("c3", "sawtooth", "none"): (404743680, 115918336),
+    ("c4", "cyclic", "mirrored"): (967579136, 251989504),
+    ("c4", "sawtooth", "mirrored"): (948634368, 251035392),
+    ("c4", "cyclic", "none"): (1298544896, 259954176),
+    ("c4", "sawtooth", "none"): (1721025024, 258340608),
+    ("c5", "cyclic", "mirrored"): (2723122688, 523010304),
+    ("c5", "sawtooth", "mirrored"): (2680911872, 525475328),
+    ("c5", "cyclic", "none"): (5061657856, 533069312),
+    ("c5", "sawtooth", "none"): (10477283072, 532609536),
+}
 
 
 def measured_peaks():
@@ -326,13 +337,16 @@ class Bench:
         clk["kernel_mhz"] = legs[headline]["kernel_mhz"]
         peaks = measured_peaks()
         tf_head = w.flops / ms_head / 1e9
+        pairing_name = {1: "none", 2: "mirrored", 3: "adjacent"}[plan.pairing]
+        default_plan = self.args.max_ctas == 0 and self.args.digit_order == "tile"
+        dram = NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, headline, pairing_name)) if default_plan else None
         # Which measured peak the run is compared with: the launches ran one after the other for the warm-up load and the
         # timed region, i.e. as a sustained, power-capped load, when the kernel's own clock sat under 80 % of the maximum.
         capped = bool(clk.get("sm_max_mhz")) and legs[headline]["kernel_mhz"] < 0.8 * clk["sm_max_mhz"]
         peak_kind = "sustained" if capped else "burst"
         block = {
             "config": config_of(w, {"scan_order": headline, "grid": plan.grid, "rows_per_item": plan.rows_per_item, "block_n": plan.block_n,
-                                    "kv_stages": plan.kv_stages, "pairing": {1: "none", 2: "mirrored", 3: "adjacent"}[plan.pairing],
+                                    "kv_stages": plan.kv_stages, "pairing": pairing_name,
                                     "timing": f"{len(seq)} scan orders launched in alternation, per-launch CUDA events, {rounds} warm-up rounds"}),
             "ms_per_step": ms_head, "ms_per_step_median": float(np.median(per_order[headline])), "tflops": tf_head,
             "orders": {o: {"ms_mean": float(np.mean(v)), "ms_median": float(np.median(v)), "tflops": w.flops / float(np.mean(v)) / 1e9,
@@ -347,7 +361,9 @@ class Bench:
                          "frac_of_clock_scaled_peak": legs[headline]["frac_of_clock_scaled_peak"],
                          "cycles_per_kv_step": legs[headline]["cycles_per_kv_step"],
                          "flops_per_launch": w.flops, "launch_ms": ms_head,
-                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, headline)), "compulsory_bytes": w.compulsory_bytes},
+                         "traffic": (dram[0] + dram[1]) if dram else None, "compulsory_bytes": w.compulsory_bytes,
+                         "dram_read_bytes": dram[0] if dram else None, "compulsory_read_bytes": 3 * w.compulsory_bytes // 4,
+                         "read_amplification": (dram[0] / (3 * w.compulsory_bytes / 4)) if dram else None},
         }
         if len(seq) == 2:
             block["sawtooth_over_cyclic"] = float(np.mean(per_order["cyclic"]) / np.mean(per_order["sawtooth"]))

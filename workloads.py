@@ -73,6 +73,11 @@ STUDY_CASES = {
     "long-512k": Workload("long-512k", 1, 1, 524288, 128, BF16, False, 2007),
     "long-128k-b8": Workload("long-128k-b8", 8, 1, 131072, 64, F16, False, 2008),
 }
+# The batch sweep of the paper's CUDA results (batch 1, 2, 4, 8; one head; 128k keys), at the paper's head dimension
+# and at 128.
+for _b in (1, 2, 4, 8):
+    STUDY_CASES[f"sweep-d64-b{_b}"] = Workload(f"sweep-d64-b{_b}", _b, 1, 131072, 64, F16, False, 2100 + _b)
+    STUDY_CASES[f"sweep-d128-b{_b}"] = Workload(f"sweep-d128-b{_b}", _b, 1, 131072, 128, BF16, False, 2200 + _b)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
