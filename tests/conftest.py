@@ -17,10 +17,18 @@ def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
 
 
+def nvcc_available() -> bool:
+    import shutil
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    return os.path.exists(nvcc) or shutil.which(nvcc) is not None
+
+
 @pytest.fixture(scope="session", autouse=True)
 def built_libraries():
-    """The C-ABI library and the C part of the oracle are built in-tree before any test (a no-op when they are fresh)."""
-    from paper_2601_16032_b200 import build as lib_build
+    """The C part of the oracle is built in-tree before any test; so is the C-ABI library where nvcc exists (both are
+    no-ops when fresh).  Without nvcc the oracle's own pins still run; the tests that load the CUDA library skip."""
     from oracle import build as oracle_build
-    lib_build.build()
     oracle_build.build()
+    if nvcc_available():
+        from paper_2601_16032_b200 import build as lib_build
+        lib_build.build()
