@@ -183,6 +183,10 @@ int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* 
  * pipeline starts after everything already enqueued on `stream` and `stream` waits for its end, so to the caller it
  * behaves like work enqueued on `stream`.  Returns without waiting: o_host is valid once `stream` has been
  * synchronised.  The first pipelined call on a device creates the streams and events (no device memory).
+ * Every argument and option is checked before the first copy is enqueued; if a CUDA call fails later, `stream` is still
+ * made to wait for whatever the side streams were given.  The per-device pipeline is shared: calls from several host
+ * threads (or on several caller streams) are enqueued one after the other under a lock and their pipelines run one
+ * after the other on the side streams.  opts->lse is ignored, opts->check_mode must be 0.
  */
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
                   void* q_dev, void* k_dev, void* v_dev, void* o_dev,

@@ -1,0 +1,92 @@
+// Measuring aid: SM cycles per tcgen05.mma (kind::f16, bf16 operands, fp32 accumulate, M = 128, K = 16) as the attention
+// kernel issues them, for N = 128 and 64, with both operands in shared memory (the form of S = Q K^T) and with A in
+// tensor memory (the form of O += P V), issued by one to four threads of a CTA at once, one CTA per SM.
+//
+//     nvcc -std=c++17 -O3 -gencode arch=compute_100a,code=sm_100a -o profile_mma_rate profile_mma_rate.cu && ./profile_mma_rate
+//
+// Operands are zero-filled shared memory laid out like the kernel's tiles (128-byte swizzle, K-major); the products are
+// discarded.  Every wait is bounded; a wait that runs out shows as "status 1".
+#include <cstdio>
+#include <cstdlib>
+
+#include "paper_2601_16032_b200/csrc/ptx.cuh"
+using namespace sawtooth;
+
+constexpr int kThreads = 160;          // warp 0 owns the TMEM allocation, warps 1..4 issue
+constexpr int kSmemBytes = 96 * 1024;  // A: 2 chunks of 128 rows x 128 bytes; B: up to 256 rows
+
+__global__ void __launch_bounds__(kThreads, 1) mma_rate(int n_cols, int a_in_tmem, int batches, int issuers, unsigned long long* out, int* status) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t done[4];
+    __shared__ uint32_t tmem_base;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < kSmemBytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) ptx::mbar_init(&done[i], 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    ptx::fence_proxy_async_smem();
+    if (warp == 0) { ptx::tmem_alloc(&tmem_base, 512); ptx::tmem_relinquish(); }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = tmem_base;
+    if (warp >= 1 && warp <= issuers && ptx::elect_one()) {
+        const int me = warp - 1;
+        const uint32_t base = ptx::smem_u32(smem);
+        const uint64_t a_desc = ptx::smem_desc_sw128(base, 16, 1024);
+        const uint64_t b_desc = ptx::smem_desc_sw128(base + 32768, 16, 1024);
+        const uint32_t idesc = ptx::instr_desc_f16(1, 0, 128, (uint32_t)n_cols);
+        const long long t0 = clock64();
+        for (int it = 0; it < batches; ++it) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {   // eight K steps accumulating into this thread's own 128 columns
+                const int c = i >> 2, kk = i & 3;
+                const uint64_t ad = a_desc + (uint64_t)((c * 16384 + kk * 32) >> 4);
+                const uint64_t bd = b_desc + (uint64_t)((c * 16384 + kk * 32) >> 4);
+                const uint32_t d = tmem + me * 128;
+                if (a_in_tmem) ptx::mma_ts(d, tmem + ((me + 1) & 3) * 128 + i * 8, bd, idesc, 1);
+                else ptx::mma_ss(d, ad, bd, idesc, 1);
+            }
+        }
+        ptx::mma_commit(&done[me]);
+        const bool ok = ptx::mbar_wait(&done[me], 0, &abort_flag, 1);
+        const long long t1 = clock64();
+        if (blockIdx.x == 0 && me == 0) out[0] = (unsigned long long)(t1 - t0);
+        if (!ok) atomicExch(status, 1);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) { ptx::tc_fence_after(); ptx::tmem_dealloc(tmem, 512); }
+}
+
+int main() {
+    unsigned long long* out;
+    int* status;
+    if (cudaMalloc(&out, 8) != cudaSuccess || cudaMalloc(&status, 4) != cudaSuccess) { printf("no CUDA device\n"); return 1; }
+    cudaMemset(status, 0, 4);
+    cudaFuncSetAttribute(mma_rate, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    int sms = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
+    const int batches = 2000;
+    printf("cycles per 128 x N x 16 MMA (all issuing threads together), %d CTAs\n", sms);
+    for (int a_in_tmem = 0; a_in_tmem < 2; ++a_in_tmem)
+        for (int n : {128, 64})
+            for (int issuers = 1; issuers <= 4; ++issuers) {
+                for (int rep = 0; rep < 2; ++rep) {
+                    mma_rate<<<sms, kThreads, kSmemBytes>>>(n, a_in_tmem, batches, issuers, out, status);
+                    cudaError_t e = cudaDeviceSynchronize();
+                    if (e != cudaSuccess) { printf("error %s\n", cudaGetErrorString(e)); return 1; }
+                }
+                unsigned long long cycles = 0;
+                int st = 0;
+                cudaMemcpy(&cycles, out, 8, cudaMemcpyDeviceToHost);
+                cudaMemcpy(&st, status, 4, cudaMemcpyDeviceToHost);
+                const double per = (double)cycles / (8.0 * batches * issuers);
+                printf("A in %s, N = %3d, %d issuing thread(s): %6.1f cycles per MMA, %5.0f FLOP/clk/SM (status %d)\n",
+                       a_in_tmem ? "TMEM" : "smem", n, issuers, per, 2.0 * 128 * n * 16 / per, st);
+            }
+    return 0;
+}
