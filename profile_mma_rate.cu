@@ -15,6 +15,8 @@ using namespace sawtooth;
 constexpr int kThreads = 160;          // warp 0 owns the TMEM allocation, warps 1..4 issue
 constexpr int kSmemBytes = 96 * 1024;  // A: 2 chunks of 128 rows x 128 bytes; B: up to 256 rows
 
+// a_in_tmem: 0 = every MMA takes A from shared memory, 1 = from tensor memory, 2 = a thread alternates the two forms,
+// 3 = even issuing threads use shared memory, odd ones tensor memory.
 __global__ void __launch_bounds__(kThreads, 1) mma_rate(int n_cols, int a_in_tmem, int batches, int issuers, unsigned long long* out, int* status) {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ uint64_t done[4];
@@ -46,8 +48,10 @@ __global__ void __launch_bounds__(kThreads, 1) mma_rate(int n_cols, int a_in_tme
                 const int c = i >> 2, kk = i & 3;
                 const uint64_t ad = a_desc + (uint64_t)((c * 16384 + kk * 32) >> 4);
                 const uint64_t bd = b_desc + (uint64_t)((c * 16384 + kk * 32) >> 4);
-                const uint32_t d = tmem + me * 128;
-                if (a_in_tmem) ptx::mma_ts(d, tmem + ((me + 1) & 3) * 128 + i * 8, bd, idesc, 1);
+                const bool from_tmem = a_in_tmem == 1 || (a_in_tmem == 2 && (i & 1)) || (a_in_tmem == 3 && (me & 1));
+                // The two forms of a mix accumulate into columns of their own: 256 columns per thread then (at most two threads).
+                const uint32_t d = a_in_tmem == 2 ? tmem + me * 256 + (i & 1) * 128 : tmem + me * 128;
+                if (from_tmem) ptx::mma_ts(d, tmem + ((me + 1) & 3) * 128 + i * 8, bd, idesc, 1);
                 else ptx::mma_ss(d, ad, bd, idesc, 1);
             }
         }
@@ -72,9 +76,10 @@ int main() {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
     const int batches = 2000;
     printf("cycles per 128 x N x 16 MMA (all issuing threads together), %d CTAs\n", sms);
-    for (int a_in_tmem = 0; a_in_tmem < 2; ++a_in_tmem)
+    for (int a_in_tmem = 0; a_in_tmem < 4; ++a_in_tmem)
         for (int n : {128, 64})
             for (int issuers = 1; issuers <= 4; ++issuers) {
+                if (a_in_tmem == 2 && issuers > 2) continue;   // 256 columns per thread
                 for (int rep = 0; rep < 2; ++rep) {
                     mma_rate<<<sms, kThreads, kSmemBytes>>>(n, a_in_tmem, batches, issuers, out, status);
                     cudaError_t e = cudaDeviceSynchronize();
@@ -85,8 +90,9 @@ int main() {
                 cudaMemcpy(&cycles, out, 8, cudaMemcpyDeviceToHost);
                 cudaMemcpy(&st, status, 4, cudaMemcpyDeviceToHost);
                 const double per = (double)cycles / (8.0 * batches * issuers);
+                const char* where[4] = {"smem", "TMEM", "smem and TMEM alternating in each thread", "smem (even threads) / TMEM (odd threads)"};
                 printf("A in %s, N = %3d, %d issuing thread(s): %6.1f cycles per MMA, %5.0f FLOP/clk/SM (status %d)\n",
-                       a_in_tmem ? "TMEM" : "smem", n, issuers, per, 2.0 * 128 * n * 16 / per, st);
+                       where[a_in_tmem], n, issuers, per, 2.0 * 128 * n * 16 / per, st);
             }
     return 0;
 }
