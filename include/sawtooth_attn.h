@@ -18,7 +18,8 @@
  * in L2.  Both orders give the same result up to the rounding order of the running sums.
  *
  * Layout: q, k, v, o are contiguous row-major [B, H, N, d] arrays (d fastest) of 16-bit elements,
- * all of the same type (IEEE fp16 or bfloat16); N_q = N_k = N.  Products accumulate in fp32; the
+ * all of the same type (IEEE fp16 or bfloat16); N_q = N_k = N.  (With opts->kv_heads set, k and v are
+ * [B, kv_heads, N, d] and groups of H / kv_heads query heads share a K/V head.)  Products accumulate in fp32; the
  * probabilities are rounded to the 16-bit type before the second product; O is rounded once at the
  * end.  Supported: d in {64, 128}; any B, H, N >= 1 with B*H <= 2^31-1 and N <= 2^24; scale finite
  * (any sign; zero gives every visible key the same weight).  Every base pointer must be 16-byte aligned.  `o` must
@@ -83,7 +84,9 @@ typedef struct {
     int pairing;      /* attn_pairing: whether one trip of a CTA's loop takes one work item or a pair of them (see below) */
     int check_mode;   /* 1: the call waits for the device and returns ATTN_ERR_DEVICE_TIMEOUT itself if a bounded wait inside
                          its kernel (or an earlier one on the device) ran out; 0: asynchronous, poll attn_device_status */
-    int reserved[4];
+    int kv_heads;     /* grouped-query attention (outside the paper): k and v hold [B, kv_heads, N, d], kv_heads divides H, and query
+                         head h attends to K/V head h / (H / kv_heads).  0 = H (every query head has its own K/V head) */
+    int reserved[3];
 } attn_fwd_opts;
 
 /* What a call with these arguments will launch; lets a caller predict L2 traffic. */

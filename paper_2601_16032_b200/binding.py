@@ -27,7 +27,7 @@ class Opts(ctypes.Structure):
         ("max_ctas", ctypes.c_int), ("kv_stages", ctypes.c_int), ("block_n", ctypes.c_int),
         ("q_tiles", ctypes.c_int), ("digit_order", ctypes.c_int), ("launch_mode", ctypes.c_int),
         ("l2_policy", ctypes.c_int), ("host_chunks", ctypes.c_int), ("lse", ctypes.c_void_p), ("pairing", ctypes.c_int), ("check_mode", ctypes.c_int),
-        ("reserved", ctypes.c_int * 4),
+        ("kv_heads", ctypes.c_int), ("reserved", ctypes.c_int * 3),
     ]
 
 
@@ -187,8 +187,9 @@ def forward(q, k, v, causal: bool = False, scan_order: int = SAWTOOTH, scale: Op
         raise AttnError(-1, "q, k and v must be CUDA tensors")
     if q.dtype not in (torch.float16, torch.bfloat16) or k.dtype != q.dtype or v.dtype != q.dtype:
         raise AttnError(-1, "q, k and v must share dtype float16 or bfloat16")
-    if q.dim() != 4 or k.shape != q.shape or v.shape != q.shape:
-        raise AttnError(-1, "q, k and v must be [B, H, N, d] of one shape")
+    if q.dim() != 4 or k.dim() != 4 or v.shape != k.shape or k.shape[0] != q.shape[0] or k.shape[2:] != q.shape[2:] or \
+            q.shape[1] % k.shape[1] != 0:
+        raise AttnError(-1, "q must be [B, H, N, d], k and v [B, H_kv, N, d] with H_kv dividing H")
     if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
         raise AttnError(-1, "q, k and v must be contiguous")
     B, H, N, d = q.shape
@@ -198,6 +199,10 @@ def forward(q, k, v, causal: bool = False, scan_order: int = SAWTOOTH, scale: Op
         raise AttnError(-1, "out must match q")
     if scale is None:
         scale = 1.0 / float(d) ** 0.5
+    if k.shape[1] != H:   # grouped-query attention: fewer K/V heads than query heads
+        import copy
+        opts = copy.copy(opts) if opts is not None else Opts()
+        opts.kv_heads = int(k.shape[1])
     stream = torch.cuda.current_stream(q.device).cuda_stream
     with torch.cuda.device(q.device):
         attn_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), B, H, N, d, float(scale), int(causal),

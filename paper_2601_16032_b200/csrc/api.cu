@@ -52,7 +52,7 @@ DeviceState g_device[kMaxDevices];
 std::mutex g_device_mutex;
 
 struct Resolved {
-    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas, pairing, check_mode;
+    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas, pairing, check_mode, kv_heads;
     size_t smem;
 };
 
@@ -71,7 +71,7 @@ int check_shape(int B, int H, int N, int d, int causal, int dtype) {
 }
 
 // `dynamic`: the call uses the dynamic schedule (items are claimed one by one, so there are no pairs).
-int resolve_opts(const attn_fwd_opts* o, int d, int causal, bool dynamic, int smem_limit, Resolved* r) {
+int resolve_opts(const attn_fwd_opts* o, int d, int H, int causal, bool dynamic, int smem_limit, Resolved* r) {
     attn_fwd_opts z;
     memset(&z, 0, sizeof(z));
     if (o) z = *o;
@@ -93,6 +93,9 @@ int resolve_opts(const attn_fwd_opts* o, int d, int causal, bool dynamic, int sm
                : z.pairing == ATTN_PAIR_DEFAULT ? (causal ? kPairMirrored : kPairNone)
                : z.pairing == ATTN_PAIR_NONE ? kPairNone : z.pairing == ATTN_PAIR_MIRRORED ? kPairMirrored : kPairAdjacent;
     r->check_mode = z.check_mode;
+    if (z.kv_heads < 0 || (z.kv_heads > 0 && (z.kv_heads > H || H % z.kv_heads != 0)))
+        return fail(ATTN_ERR_INVALID_ARG, "kv_heads (%d) must divide the number of query heads (%d)", z.kv_heads, H);
+    r->kv_heads = z.kv_heads ? z.kv_heads : H;
     r->head_fastest = z.digit_order == ATTN_HEAD_FASTEST;
     r->launch_mode = z.launch_mode;
     r->l2_policy = z.l2_policy;
@@ -190,10 +193,10 @@ int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, i
 // thread built are kept, so that a caller who launches on the same buffers again and again pays for the encoding once.
 struct MapKey {
     const void *q, *k, *v, *o;
-    int BH, N, d, dtype, block_n, stage_rows;
+    int BH, BH_kv, N, d, dtype, block_n, stage_rows;
     bool operator==(const MapKey& x) const {
-        return q == x.q && k == x.k && v == x.v && o == x.o && BH == x.BH && N == x.N && d == x.d && dtype == x.dtype &&
-               block_n == x.block_n && stage_rows == x.stage_rows;
+        return q == x.q && k == x.k && v == x.v && o == x.o && BH == x.BH && BH_kv == x.BH_kv && N == x.N && d == x.d &&
+               dtype == x.dtype && block_n == x.block_n && stage_rows == x.stage_rows;
     }
 };
 struct MapSet { MapKey key; CUtensorMap tq, tk, tv, to; bool valid = false; };
@@ -208,8 +211,8 @@ int maps_for(const MapKey& key, const MapSet** out) {
     m.valid = false;
     int rc;
     if ((rc = make_map(&m.tq, key.q, key.BH, key.N, key.d, kBlockM, key.dtype))) return rc;
-    if ((rc = make_map(&m.tk, key.k, key.BH, key.N, key.d, key.block_n, key.dtype))) return rc;
-    if ((rc = make_map(&m.tv, key.v, key.BH, key.N, key.d, key.block_n, key.dtype))) return rc;
+    if ((rc = make_map(&m.tk, key.k, key.BH_kv, key.N, key.d, key.block_n, key.dtype))) return rc;
+    if ((rc = make_map(&m.tv, key.v, key.BH_kv, key.N, key.d, key.block_n, key.dtype))) return rc;
     // O is written through shared memory in boxes of 64 columns x as many rows as one warp's share of a ring slot holds.
     if ((rc = make_map(&m.to, key.o, key.BH, key.N, key.d, key.stage_rows, key.dtype))) return rc;
     m.key = key;
@@ -303,7 +306,7 @@ int attn_query_plan(int B, int H, int N, int d, int causal, int dtype, const att
         smem_limit = ds.smem_optin;
     }
     Resolved r;
-    rc = resolve_opts(opts, d, causal, false, smem_limit, &r);
+    rc = resolve_opts(opts, d, H, causal, false, smem_limit, &r);
     if (rc) return rc;
     const SchedParams sp = make_sched(B, H, N, r.q_tiles, r.block_n, causal, 0, r.head_fastest, 0, r.pairing);
     out->block_m = kBlockM;
@@ -416,7 +419,7 @@ static int check_call(const void* q, const void* k, const void* v, void* o, int 
     if (opts && opts->lse && ((uintptr_t)opts->lse & 3u)) return fail(ATTN_ERR_ALIGNMENT, "opts->lse must be 4-byte aligned");
     rc = current_device(&c->ds, &c->dev);
     if (rc) return rc;
-    return resolve_opts(opts, d, causal, dynamic, c->ds.smem_optin, &c->r);
+    return resolve_opts(opts, d, H, causal, dynamic, c->ds.smem_optin, &c->r);
 }
 
 static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
@@ -439,6 +442,7 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
     kp.scale_log2 = mag * 1.4426950408889634f;
     kp.negate = scale < 0.f;
     kp.kv_stages = r.stages;
+    kp.kv_heads = r.kv_heads;
     kp.l2_policy = r.l2_policy;
     kp.o = o;
     kp.lse = opts ? opts->lse : nullptr;
@@ -447,7 +451,7 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
 
     MapKey key;
     key.q = q; key.k = k; key.v = v; key.o = o;
-    key.BH = B * H; key.N = N; key.d = d; key.dtype = dtype; key.block_n = r.block_n;
+    key.BH = B * H; key.BH_kv = B * r.kv_heads; key.N = N; key.d = d; key.dtype = dtype; key.block_n = r.block_n;
     key.stage_rows = (r.block_n * d * 2 / 2 / 4) / 128 < 32 ? (r.block_n * d * 2 / 2 / 4) / 128 : 32;
     const MapSet* maps = nullptr;
     if ((rc = maps_for(key, &maps))) return rc;
@@ -515,6 +519,7 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     int rc = check_call(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, opts, false, &c);
     if (rc) return rc;
     if (c.r.check_mode) return fail(ATTN_ERR_INVALID_ARG, "check_mode would make attn_fwd_host wait inside its pipeline: call attn_device_status afterwards instead");
+    if (c.r.kv_heads != H) return fail(ATTN_ERR_UNSUPPORTED, "attn_fwd_host cuts the heads into groups and takes as many K/V heads as query heads (kv_heads = 0)");
     attn_fwd_opts inner;
     memset(&inner, 0, sizeof(inner));
     if (opts) inner = *opts;

@@ -40,6 +40,7 @@ struct KernelParams {
     SchedParams sched;
     float scale_log2;     // |scale| * log2(e): probabilities are computed with ex2
     int negate;           // 1: scale < 0, the scores change sign before anything else is done with them
+    int kv_heads;         // K/V heads per batch entry; query head h reads K/V head h / (H / kv_heads)
     int kv_stages;        // slots in the K/V ring
     int l2_policy;        // 1: K/V loads evict_last, Q loads evict_first
     void* o;              // [B, H, N, d] output
@@ -283,6 +284,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             __syncwarp();
             ++q_issued;
+            // Grouped-query attention: the H / kv_heads query heads of a group stream the same K/V head.
+            const int bh_kv = (w.bh / p.sched.H) * p.kv_heads + (w.bh % p.sched.H) / (p.sched.H / p.kv_heads);
             for (int s = 0; ok && s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
                 for (int kv = 0; kv < 2; ++kv) {
@@ -294,8 +297,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                         for (int c = 0; c < G::kChunks; ++c) {
                             void* dst = kv_smem + (size_t)ring.slot * G::kKVTileBytes + c * G::kKVChunkBytes;
-                            if (p.l2_policy) ptx::tma_load_3d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh, pol_kv);
-                            else ptx::tma_load_3d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, w.bh);
+                            if (p.l2_policy) ptx::tma_load_3d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, bh_kv, pol_kv);
+                            else ptx::tma_load_3d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, bh_kv);
                         }
                     }
                     __syncwarp();
@@ -440,8 +443,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (!ok) break;
                 if (hi_mine > 0) ptx::mma_commit(&bar->o_full[q]);
-                // The staging slot is released by the tile's softmax warps, or here if the tile lies beyond N.
-                if (hi_mine == 0) ptx::mbar_arrive(&bar->kv_empty[ring.slot]);
+                // The item's staging slot is not this lane's business: the softmax warps take it over from the producer
+                // and hand it back.  (A lane whose tile lies beyond N has nothing to wait for in an item and may be a whole
+                // item ahead of the softmax warps, so it must not count towards that slot's release.)
                 ring.advance(stages);
             }
             // Nothing of this thread's MMAs may be in flight when TMEM is released.
@@ -668,7 +672,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (lane == 0) ptx::mbar_arrive(&bar->stage_done[q]);
             if ((warp & 3) == 0) {
                 ok = ptx::warp_all(ptx::mbar_wait(&bar->stage_done[q], stage_phase, abort_flag, kSiteStageDone));
-                if (ok && lane == 0) ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
+                // One arrival per Q tile of the item; a second tile that lies beyond N has no warps at work: the first
+                // tile's warp arrives for it, after its own rows have left the slot.
+                if (ok && lane == 0) {
+                    ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
+                    if (kQTiles == 2 && q == 0 && w.hi_q[1] == 0) ptx::mbar_arrive(&bar->kv_empty[stage.slot]);
+                }
             }
             stage_phase ^= 1u;
             if (!ok) break;

@@ -293,3 +293,34 @@ def test_repeated_calls_reuse_cached_tensor_maps_correctly():
     err = np.abs(f(o) - ora.attention_head(f(qc), f(kc), f(vc), wc.scale, True))
     assert err.max() <= 2e-2 and err.mean() <= 2e-3
     assert torch.equal(run_cuda(wa, a, sa.CYCLIC), want_a)
+
+
+@pytest.mark.parametrize("N", [1, 100, 128])
+@pytest.mark.parametrize("kv_stages", [0, 3])
+def test_many_one_tile_items_per_cta(N, kv_stages):
+    """Heads of at most 128 rows: the second Q tile of every work item lies beyond N, so its MMA lane has nothing to wait for
+    and runs ahead of the softmax warps, item after item.  Few CTAs, many items each, repeated launches, static and
+    dynamic schedule: the staging slot of the ring must be handed back by the warps that used it, not by that lane."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("tiny-items", 4, 8, N, 64, wl.BF16, False, 7700 + N)
+    qkv = upload(w)
+    q, k, v = qkv
+    opts = opts_for(kv_stages=kv_stages, max_ctas=2, block_n=64)
+    want = None
+    for rep in range(10):
+        o = run_cuda(w, qkv, sa.SAWTOOTH if rep % 2 else sa.CYCLIC, opts)
+        if want is None:
+            assert_parity(w, o)
+            want = o
+        else:
+            assert torch.equal(o.view(torch.int16), want.view(torch.int16))
+    dyn = opts_for(kv_stages=kv_stages, max_ctas=2, block_n=64, pairing=1)
+    nb = sa.attn_dynamic_scratch_bytes(2)
+    scratch = torch.zeros(nb // 4, dtype=torch.int32, device=q.device)
+    for rep in range(10):
+        o = torch.full_like(q, float("nan"))
+        sa.attn_fwd_dynamic(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, 0, sa.CYCLIC, sa.BF16,
+                            torch.cuda.current_stream().cuda_stream, dyn, scratch.data_ptr(), nb)
+        sa.attn_device_status()
+        assert torch.equal(o.view(torch.int16), want.view(torch.int16))
