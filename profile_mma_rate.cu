@@ -66,6 +66,74 @@ __global__ void __launch_bounds__(kThreads, 1) mma_rate(int n_cols, int a_in_tme
     if (warp == 0) { ptx::tc_fence_after(); ptx::tmem_dealloc(tmem, 512); }
 }
 
+// The same measurement for the two-SM form (cta_group::2): a cluster of two CTAs, M = 256 (128 rows in each CTA's tensor
+// memory), N = 128 with each CTA holding 64 of the 128 B rows in its own shared memory; one thread of the cluster's first
+// CTA issues for both.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+mma_rate_pair(int a_in_tmem, int batches, unsigned long long* out, int* status) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t done;
+    __shared__ uint32_t tmem_base;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < kSmemBytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) { ptx::mbar_init(&done, 1); abort_flag = 0; ptx::fence_mbar_init(); }
+    ptx::fence_proxy_async_smem();
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(&tmem_base)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    ptx::tc_fence_after();
+    const uint32_t tmem = tmem_base;
+    if (cluster_rank() == 0 && warp == 1 && ptx::elect_one()) {
+        const uint32_t base = ptx::smem_u32(smem);
+        const uint64_t a_desc = ptx::smem_desc_sw128(base, 16, 1024);
+        const uint64_t b_desc = ptx::smem_desc_sw128(base + 32768, 16, 1024);
+        const uint32_t idesc = ptx::instr_desc_f16(1, 0, 256, 128);
+        const long long t0 = clock64();
+        for (int it = 0; it < batches; ++it) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int c = i >> 2, kk = i & 3;
+                const uint64_t ad = a_desc + (uint64_t)((c * 16384 + kk * 32) >> 4);
+                const uint64_t bd = b_desc + (uint64_t)((c * 8192 + kk * 32) >> 4);
+                if (a_in_tmem)
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                                 ::"r"(tmem), "r"(tmem + 256 + i * 8), "l"(bd), "r"(idesc), "r"(1u) : "memory");
+                else
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                 ::"r"(tmem), "l"(ad), "l"(bd), "r"(idesc), "r"(1u) : "memory");
+            }
+        }
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(ptx::smem_u32(&done)) : "memory");
+        const bool ok = ptx::mbar_wait(&done, 0, &abort_flag, 1);
+        const long long t1 = clock64();
+        if (blockIdx.x == 0) out[0] = (unsigned long long)(t1 - t0);
+        if (!ok) atomicExch(status, 1);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 0) {
+        ptx::tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
 int main() {
     unsigned long long* out;
     int* status;
@@ -94,5 +162,20 @@ int main() {
                 printf("A in %s, N = %3d, %d issuing thread(s): %6.1f cycles per MMA, %5.0f FLOP/clk/SM (status %d)\n",
                        where[a_in_tmem], n, issuers, per, 2.0 * 128 * n * 16 / per, st);
             }
+    cudaFuncSetAttribute(mma_rate_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    for (int a_in_tmem = 0; a_in_tmem < 2; ++a_in_tmem) {
+        for (int rep = 0; rep < 2; ++rep) {
+            mma_rate_pair<<<sms & ~1, kThreads, kSmemBytes>>>(a_in_tmem, batches, out, status);
+            cudaError_t e = cudaDeviceSynchronize();
+            if (e != cudaSuccess) { printf("error %s\n", cudaGetErrorString(e)); return 1; }
+        }
+        unsigned long long cycles = 0;
+        int st = 0;
+        cudaMemcpy(&cycles, out, 8, cudaMemcpyDeviceToHost);
+        cudaMemcpy(&st, status, 4, cudaMemcpyDeviceToHost);
+        const double per = (double)cycles / (8.0 * batches);
+        printf("two SMs (cta_group::2), M = 256, N = 128, A in %s, 1 issuing thread: %6.1f cycles per MMA, %5.0f FLOP/clk/SM (status %d)\n",
+               a_in_tmem ? "TMEM" : "smem", per, 2.0 * 128 * 128 * 16 / per, st);
+    }
     return 0;
 }
