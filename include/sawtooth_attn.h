@@ -19,7 +19,8 @@
  *
  * Layout: q, k, v, o are contiguous row-major [B, H, N, d] arrays (d fastest) of 16-bit elements,
  * all of the same type (IEEE fp16 or bfloat16); N_q = N_k = N.  (With opts->kv_heads set, k and v are
- * [B, kv_heads, N, d] and groups of H / kv_heads query heads share a K/V head.)  Products accumulate in fp32; the
+ * [B, kv_heads, N, d] and groups of H / kv_heads query heads share a K/V head; with opts->layout =
+ * ATTN_LAYOUT_BNHD all four are [B, N, heads, d].)  Products accumulate in fp32; the
  * probabilities are rounded to the 16-bit type before the second product; O is rounded once at the
  * end.  Supported: d in {64, 128}; any B, H, N >= 1 with B*H <= 2^31-1 and N <= 2^24; scale finite
  * (any sign; zero gives every visible key the same weight).  Every base pointer must be 16-byte aligned.  `o` must
@@ -55,6 +56,7 @@ typedef enum {
 typedef enum { ATTN_SCAN_CYCLIC = 0, ATTN_SCAN_SAWTOOTH = 1 } attn_scan_order;
 typedef enum { ATTN_F16 = 0, ATTN_BF16 = 1 } attn_dtype;
 typedef enum { ATTN_TILE_FASTEST = 0, ATTN_HEAD_FASTEST = 1 } attn_digit_order;
+typedef enum { ATTN_LAYOUT_BHND = 0, ATTN_LAYOUT_BNHD = 1 } attn_layout;
 /*
  * How the static walk of Algorithm 2 groups work items.  With pairs, a unit of the walk is two W-row Q blocks of one
  * head which the CTA handles one after the other, the first scanned first-to-last and, in the sawtooth order, the
@@ -86,7 +88,9 @@ typedef struct {
                          its kernel (or an earlier one on the device) ran out; 0: asynchronous, poll attn_device_status */
     int kv_heads;     /* grouped-query attention (outside the paper): k and v hold [B, kv_heads, N, d], kv_heads divides H, and query
                          head h attends to K/V head h / (H / kv_heads).  0 = H (every query head has its own K/V head) */
-    int reserved[3];
+    int layout;       /* attn_layout of q, k, v and o (outside the paper): ATTN_LAYOUT_BHND = [B, H, N, d] (default), ATTN_LAYOUT_BNHD =
+                         [B, N, H, d], the order in which projection layers leave them.  lse stays [B, H, N]. */
+    int reserved[2];
 } attn_fwd_opts;
 
 /* What a call with these arguments will launch; lets a caller predict L2 traffic. */

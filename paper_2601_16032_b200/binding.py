@@ -9,6 +9,7 @@ CYCLIC, SAWTOOTH = 0, 1
 F16, BF16 = 0, 1
 TILE_FASTEST, HEAD_FASTEST = 0, 1
 PAIR_DEFAULT, PAIR_NONE, PAIR_MIRRORED, PAIR_ADJACENT = 0, 1, 2, 3
+LAYOUT_BHND, LAYOUT_BNHD = 0, 1
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libsawtooth_attn.so")
@@ -27,7 +28,7 @@ class Opts(ctypes.Structure):
         ("max_ctas", ctypes.c_int), ("kv_stages", ctypes.c_int), ("block_n", ctypes.c_int),
         ("q_tiles", ctypes.c_int), ("digit_order", ctypes.c_int), ("launch_mode", ctypes.c_int),
         ("l2_policy", ctypes.c_int), ("host_chunks", ctypes.c_int), ("lse", ctypes.c_void_p), ("pairing", ctypes.c_int), ("check_mode", ctypes.c_int),
-        ("kv_heads", ctypes.c_int), ("reserved", ctypes.c_int * 3),
+        ("kv_heads", ctypes.c_int), ("layout", ctypes.c_int), ("reserved", ctypes.c_int * 2),
     ]
 
 

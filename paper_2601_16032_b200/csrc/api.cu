@@ -52,7 +52,7 @@ DeviceState g_device[kMaxDevices];
 std::mutex g_device_mutex;
 
 struct Resolved {
-    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas, pairing, check_mode, kv_heads;
+    int block_n, q_tiles, stages, head_fastest, launch_mode, l2_policy, max_ctas, pairing, check_mode, kv_heads, layout;
     size_t smem;
 };
 
@@ -96,6 +96,8 @@ int resolve_opts(const attn_fwd_opts* o, int d, int H, int causal, bool dynamic,
     if (z.kv_heads < 0 || (z.kv_heads > 0 && (z.kv_heads > H || H % z.kv_heads != 0)))
         return fail(ATTN_ERR_INVALID_ARG, "kv_heads (%d) must divide the number of query heads (%d)", z.kv_heads, H);
     r->kv_heads = z.kv_heads ? z.kv_heads : H;
+    if (z.layout != ATTN_LAYOUT_BHND && z.layout != ATTN_LAYOUT_BNHD) return fail(ATTN_ERR_INVALID_ARG, "unknown layout %d", z.layout);
+    r->layout = z.layout;
     r->head_fastest = z.digit_order == ATTN_HEAD_FASTEST;
     r->launch_mode = z.launch_mode;
     r->l2_policy = z.l2_policy;
@@ -173,16 +175,20 @@ int get_encoder(EncodeTiledFn* fn) {
     return ATTN_OK;
 }
 
-// [B*H, N, d] view, box = 64 columns x `rows` rows of one head, 128-byte swizzle, zero fill outside.
-int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, int dtype) {
+// [B, heads, N, d] view of a tensor stored as [B, heads, N, d] (layout 0) or [B, N, heads, d] (layout 1); dimensions from
+// the innermost: d, N, heads, B.  Box = 64 columns x `rows` rows of one head, 128-byte swizzle, zero fill outside.
+int make_map(CUtensorMap* m, const void* base, int B, int heads, int N, int d, int rows, int dtype, int layout) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc) return rc;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(m, dtype == ATTN_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)heads, (cuuint64_t)B};
+    const cuuint64_t row = (cuuint64_t)d * 2;
+    cuuint64_t strides[3];
+    if (layout == 0) { strides[0] = row; strides[1] = row * N; strides[2] = row * N * heads; }
+    else { strides[0] = row * heads; strides[1] = row; strides[2] = row * heads * N; }
+    cuuint32_t box[4] = {64, (cuuint32_t)rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(m, dtype == ATTN_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ATTN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
@@ -193,10 +199,10 @@ int make_map(CUtensorMap* m, const void* base, int BH, int N, int d, int rows, i
 // thread built are kept, so that a caller who launches on the same buffers again and again pays for the encoding once.
 struct MapKey {
     const void *q, *k, *v, *o;
-    int BH, BH_kv, N, d, dtype, block_n, stage_rows;
+    int B, H, H_kv, N, d, dtype, block_n, stage_rows, layout;
     bool operator==(const MapKey& x) const {
-        return q == x.q && k == x.k && v == x.v && o == x.o && BH == x.BH && BH_kv == x.BH_kv && N == x.N && d == x.d &&
-               dtype == x.dtype && block_n == x.block_n && stage_rows == x.stage_rows;
+        return q == x.q && k == x.k && v == x.v && o == x.o && B == x.B && H == x.H && H_kv == x.H_kv && N == x.N && d == x.d &&
+               dtype == x.dtype && block_n == x.block_n && stage_rows == x.stage_rows && layout == x.layout;
     }
 };
 struct MapSet { MapKey key; CUtensorMap tq, tk, tv, to; bool valid = false; };
@@ -210,11 +216,11 @@ int maps_for(const MapKey& key, const MapSet** out) {
     MapSet& m = g_maps[g_maps_next];
     m.valid = false;
     int rc;
-    if ((rc = make_map(&m.tq, key.q, key.BH, key.N, key.d, kBlockM, key.dtype))) return rc;
-    if ((rc = make_map(&m.tk, key.k, key.BH_kv, key.N, key.d, key.block_n, key.dtype))) return rc;
-    if ((rc = make_map(&m.tv, key.v, key.BH_kv, key.N, key.d, key.block_n, key.dtype))) return rc;
+    if ((rc = make_map(&m.tq, key.q, key.B, key.H, key.N, key.d, kBlockM, key.dtype, key.layout))) return rc;
+    if ((rc = make_map(&m.tk, key.k, key.B, key.H_kv, key.N, key.d, key.block_n, key.dtype, key.layout))) return rc;
+    if ((rc = make_map(&m.tv, key.v, key.B, key.H_kv, key.N, key.d, key.block_n, key.dtype, key.layout))) return rc;
     // O is written through shared memory in boxes of 64 columns x as many rows as one warp's share of a ring slot holds.
-    if ((rc = make_map(&m.to, key.o, key.BH, key.N, key.d, key.stage_rows, key.dtype))) return rc;
+    if ((rc = make_map(&m.to, key.o, key.B, key.H, key.N, key.d, key.stage_rows, key.dtype, key.layout))) return rc;
     m.key = key;
     m.valid = true;
     g_maps_next = (g_maps_next + 1) % kMapCacheSize;
@@ -451,7 +457,7 @@ static int fwd_common(const void* q, const void* k, const void* v, void* o, int 
 
     MapKey key;
     key.q = q; key.k = k; key.v = v; key.o = o;
-    key.BH = B * H; key.BH_kv = B * r.kv_heads; key.N = N; key.d = d; key.dtype = dtype; key.block_n = r.block_n;
+    key.B = B; key.H = H; key.H_kv = r.kv_heads; key.layout = r.layout; key.N = N; key.d = d; key.dtype = dtype; key.block_n = r.block_n;
     key.stage_rows = (r.block_n * d * 2 / 2 / 4) / 128 < 32 ? (r.block_n * d * 2 / 2 / 4) / 128 : 32;
     const MapSet* maps = nullptr;
     if ((rc = maps_for(key, &maps))) return rc;
@@ -519,6 +525,7 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     int rc = check_call(q_dev, k_dev, v_dev, o_dev, B, H, N, d, scale, causal, scan_order, dtype, opts, false, &c);
     if (rc) return rc;
     if (c.r.check_mode) return fail(ATTN_ERR_INVALID_ARG, "check_mode would make attn_fwd_host wait inside its pipeline: call attn_device_status afterwards instead");
+    if (c.r.layout != ATTN_LAYOUT_BHND) return fail(ATTN_ERR_UNSUPPORTED, "attn_fwd_host cuts the heads into contiguous groups: layout must be ATTN_LAYOUT_BHND");
     if (c.r.kv_heads != H) return fail(ATTN_ERR_UNSUPPORTED, "attn_fwd_host cuts the heads into groups and takes as many K/V heads as query heads (kv_heads = 0)");
     attn_fwd_opts inner;
     memset(&inner, 0, sizeof(inner));

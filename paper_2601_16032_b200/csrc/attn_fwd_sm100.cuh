@@ -40,7 +40,7 @@ struct KernelParams {
     SchedParams sched;
     float scale_log2;     // |scale| * log2(e): probabilities are computed with ex2
     int negate;           // 1: scale < 0, the scores change sign before anything else is done with them
-    int kv_heads;         // K/V heads per batch entry; query head h reads K/V head h / (H / kv_heads)
+    int kv_heads;         // K/V heads per batch entry; query head h reads K/V head h / (H / kv_heads) (grouped-query attention)
     int kv_stages;        // slots in the K/V ring
     int l2_policy;        // 1: K/V loads evict_last, Q loads evict_first
     void* o;              // [B, H, N, d] output
@@ -266,6 +266,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             ok = ptx::warp_all(ptx::mbar_wait(&bar->q_empty, (it & 1) ^ 1, abort_flag, kSiteProducerQ));
             if (!ok) break;
+            // Tensor coordinates of the item's head: (batch, head) for Q, (batch, head of its group) for K and V.
+            const int b_idx = w.bh / p.sched.H, h_idx = w.bh % p.sched.H;
+            const int h_kv = h_idx / (p.sched.H / p.kv_heads);
             if (ptx::elect_one()) {
                 int n_valid = 0;
 #pragma unroll
@@ -277,15 +280,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < G::kChunks; ++c) {
                         void* dst = q_smem + q * G::kQTileBytes + c * G::kQChunkBytes;
-                        if (p.l2_policy) ptx::tma_load_3d_hint(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh, pol_q);
-                        else ptx::tma_load_3d(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, w.bh);
+                        if (p.l2_policy) ptx::tma_load_4d_hint(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, h_idx, b_idx, pol_q);
+                        else ptx::tma_load_4d(dst, &tm_q, &bar->q_full, c * 64, w.row0 + q * kBlockM, h_idx, b_idx);
                     }
                 }
             }
             __syncwarp();
             ++q_issued;
-            // Grouped-query attention: the H / kv_heads query heads of a group stream the same K/V head.
-            const int bh_kv = (w.bh / p.sched.H) * p.kv_heads + (w.bh % p.sched.H) / (p.sched.H / p.kv_heads);
             for (int s = 0; ok && s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
                 for (int kv = 0; kv < 2; ++kv) {
@@ -297,8 +298,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                         for (int c = 0; c < G::kChunks; ++c) {
                             void* dst = kv_smem + (size_t)ring.slot * G::kKVTileBytes + c * G::kKVChunkBytes;
-                            if (p.l2_policy) ptx::tma_load_3d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, bh_kv, pol_kv);
-                            else ptx::tma_load_3d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, bh_kv);
+                            if (p.l2_policy) ptx::tma_load_4d_hint(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, h_kv, b_idx, pol_kv);
+                            else ptx::tma_load_4d(dst, tm, &bar->kv_full[ring.slot], c * 64, j * kBlockN, h_kv, b_idx);
                         }
                     }
                     __syncwarp();
@@ -660,7 +661,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     __syncwarp();
                     const int y0 = tile_row0 + (warp & 3) * 32 + ps * G::kStageRows;
                     if (y0 < N && ptx::elect_one()) {   // rows of the box beyond N are dropped by the copy
-                        ptx::tma_store_3d(&tm_o, buf, c64 * 64, y0, w.bh);
+                        ptx::tma_store_4d(&tm_o, buf, c64 * 64, y0, w.bh % p.sched.H, w.bh / p.sched.H);
                         ptx::bulk_commit_group();
                         ptx::bulk_wait_group_read0();   // the buffer may be written again
                     }

@@ -87,3 +87,46 @@ def test_kv_heads_must_divide_heads_and_the_wrapper_infers_them():
     ref = torch.nn.functional.scaled_dot_product_attention(q.float(), k.float().repeat_interleave(2, dim=1), k.float().repeat_interleave(2, dim=1),
                                                            is_causal=True)
     assert (out.float() - ref).abs().max() < 2e-2
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("kv_heads", [0, 2])
+@pytest.mark.parametrize("d,dtype,N", [(128, wl.BF16, 1330), (64, wl.F16, 257)])
+def test_bnhd_layout(causal, kv_heads, d, dtype, N):
+    """q, k, v and o stored as [B, N, heads, d]: same result as the oracle head by head, log-sum-exp still [B, H, N]."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    from oracle import attention as ora
+    B, H = 2, 4
+    Hkv = kv_heads or H
+    wq = wl.small_workload("bnhd-q", B, H, N, d, dtype, causal, 7900)
+    wkv = wl.small_workload("bnhd-kv", B, Hkv, N, d, dtype, causal, 7901)
+    tdt = torch.bfloat16 if dtype == wl.BF16 else torch.float16
+
+    def up(w, name):   # [B, N, heads, d]
+        t = torch.empty((w.B, w.N, w.H, w.d), dtype=torch.int16, device="cuda:0")
+        for b, h in wl.all_heads(w):
+            t[b, :, h].copy_(torch.from_numpy(wl.head_bits(w, name, b, h).view(np.int16)))
+        return t.view(tdt)
+
+    q, k, v = up(wq, "q"), up(wkv, "k"), up(wkv, "v")
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full((B, H, N), float("nan"), dtype=torch.float32, device="cuda:0")
+    opts = sa.Opts()
+    opts.layout, opts.kv_heads, opts.max_ctas, opts.lse = sa.LAYOUT_BNHD, kv_heads, 3, lse.data_ptr()
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        sa.attn_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, wq.scale, int(causal), order,
+                       sa.BF16 if dtype == wl.BF16 else sa.F16, torch.cuda.current_stream().cuda_stream, opts)
+        sa.attn_device_status()
+        worst, total, count = 0.0, 0.0, 0
+        for b, h in wl.all_heads(wq):
+            g = h // (H // Hkv)
+            qq = wl.bits_to_f64(wl.head_bits(wq, "q", b, h), dtype)
+            kk = wl.bits_to_f64(wl.head_bits(wkv, "k", b, g), dtype)
+            vv = wl.bits_to_f64(wl.head_bits(wkv, "v", b, g), dtype)
+            got = wl.bits_to_f64(o[b, :, h].contiguous().view(torch.int16).cpu().numpy().view(np.uint16), dtype)
+            err = np.abs(got - ora.attention_head(qq, kk, vv, wq.scale, causal))
+            worst, total, count = max(worst, float(err.max())), total + float(err.sum()), count + err.size
+            want_lse = ora.logsumexp_rows(qq, np.arange(N, dtype=np.int64), kk, wq.scale, causal)
+            assert np.abs(lse[b, h].double().cpu().numpy() - want_lse).max() <= 5e-4
+        assert worst <= MAX_ABS_TOL and total / count <= MEAN_ABS_TOL, (worst, total / count)
