@@ -324,3 +324,53 @@ def test_many_one_tile_items_per_cta(N, kv_stages):
                             torch.cuda.current_stream().cuda_stream, dyn, scratch.data_ptr(), nb)
         sa.attn_device_status()
         assert torch.equal(o.view(torch.int16), want.view(torch.int16))
+
+
+def test_host_entry_point_from_two_threads():
+    """Two host threads, each with its own stream and buffers, call attn_fwd_host at the same time (ctypes drops the
+    interpreter lock during the call): the device's one pipeline is handed from call to call under its lock, and both
+    get the device entry point's result bit for bit.  The device entry point is called from both threads as well (its
+    tensor-map cache is per thread, the per-device state behind a lock)."""
+    import threading
+    import torch
+    import paper_2601_16032_b200 as sa
+    jobs = []
+    for i in range(2):
+        w = wl.small_workload(f"host-thread-{i}", 1, 6, 600 + 100 * i, 128, wl.BF16, True, 7360 + i)
+        q, k, v = upload(w)
+        want = run_cuda(w, (q, k, v), sa.CYCLIC)
+        host = [t.view(torch.int16).cpu().pin_memory() for t in (q, k, v)]
+        o_host = torch.full(q.shape, -1, dtype=torch.int16).pin_memory()
+        dev = [torch.empty_like(q) for _ in range(4)]
+        jobs.append(dict(w=w, q=q, k=k, v=v, want=want, host=host, o_host=o_host, dev=dev, stream=torch.cuda.Stream(), errors=[]))
+
+    def work(j):
+        try:
+            torch.cuda.set_device(0)
+            w = j["w"]
+            opts = sa.Opts()
+            opts.host_chunks = 3
+            for _ in range(5):
+                j["o_host"].fill_(-1)
+                sa.attn_fwd_host(j["host"][0].data_ptr(), j["host"][1].data_ptr(), j["host"][2].data_ptr(), j["o_host"].data_ptr(),
+                                 j["dev"][0].data_ptr(), j["dev"][1].data_ptr(), j["dev"][2].data_ptr(), j["dev"][3].data_ptr(),
+                                 w.B, w.H, w.N, w.d, w.scale, 1, sa.CYCLIC, sa.BF16, j["stream"].cuda_stream, opts)
+                j["stream"].synchronize()
+                if not torch.equal(j["o_host"], j["want"].view(torch.int16).cpu()):
+                    j["errors"].append("host result differs")
+                o = torch.empty_like(j["q"])
+                sa.attn_fwd(j["q"].data_ptr(), j["k"].data_ptr(), j["v"].data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, 1,
+                            sa.CYCLIC, sa.BF16, j["stream"].cuda_stream)
+                j["stream"].synchronize()
+                if not torch.equal(o, j["want"]):
+                    j["errors"].append("device result differs")
+        except Exception as e:   # surfaces in the main thread below
+            j["errors"].append(repr(e))
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    sa.attn_device_status()
+    assert all(not j["errors"] for j in jobs), [j["errors"] for j in jobs]
