@@ -52,16 +52,16 @@ WARMUP_LOAD_SECONDS = 0.25
 # kernel on the full-size workload with the default launch plan (three metrics, one pass).
 # Keyed by (workload, scan order, pairing in force); anything else reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "cyclic", "none"): (403114240, 116056576),
-    ("c3", "sawtooth", "none"): (404743680, 115918336),
-    ("c4", "cyclic", "mirrored"): (967579136, 251989504),
-    ("c4", "sawtooth", "mirrored"): (948634368, 251035392),
-    ("c4", "cyclic", "none"): (1298544896, 259954176),
-    ("c4", "sawtooth", "none"): (1721025024, 258340608),
-    ("c5", "cyclic", "mirrored"): (2723122688, 523010304),
-    ("c5", "sawtooth", "mirrored"): (2680911872, 525475328),
-    ("c5", "cyclic", "none"): (5061657856, 533069312),
-    ("c5", "sawtooth", "none"): (10477283072, 532609536),
+    ("c3", "cyclic", "none"): (406169600, 116657664),
+    ("c3", "sawtooth", "none"): (408402176, 116601600),
+    ("c4", "cyclic", "mirrored"): (978689280, 251552256),
+    ("c4", "sawtooth", "mirrored"): (974698752, 252116992),
+    ("c4", "cyclic", "none"): (1579868160, 259458816),
+    ("c4", "sawtooth", "none"): (2294563328, 257892352),
+    ("c5", "cyclic", "mirrored"): (2847872768, 526457856),
+    ("c5", "sawtooth", "mirrored"): (3283107328, 526868224),
+    ("c5", "cyclic", "none"): (6044815104, 534496512),
+    ("c5", "sawtooth", "none"): (11802469120, 531748096),
 }
 
 
