@@ -52,16 +52,16 @@ WARMUP_LOAD_SECONDS = 0.25
 # kernel on the full-size workload with the default launch plan (three metrics, one pass).
 # Keyed by (workload, scan order, pairing in force); anything else reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "cyclic", "none"): (406169600, 116657664),
-    ("c3", "sawtooth", "none"): (408402176, 116601600),
-    ("c4", "cyclic", "mirrored"): (978689280, 251552256),
-    ("c4", "sawtooth", "mirrored"): (974698752, 252116992),
-    ("c4", "cyclic", "none"): (1579868160, 259458816),
-    ("c4", "sawtooth", "none"): (2294563328, 257892352),
-    ("c5", "cyclic", "mirrored"): (2847872768, 526457856),
-    ("c5", "sawtooth", "mirrored"): (3283107328, 526868224),
-    ("c5", "cyclic", "none"): (6044815104, 534496512),
-    ("c5", "sawtooth", "none"): (11802469120, 531748096),
+    ("c3", "cyclic", "none"): (403255040, 116423936),
+    ("c3", "sawtooth", "none"): (404629248, 115891712),
+    ("c4", "cyclic", "mirrored"): (980670976, 252060416),
+    ("c4", "sawtooth", "mirrored"): (947037184, 250663424),
+    ("c4", "cyclic", "none"): (1358940928, 260275968),
+    ("c4", "sawtooth", "none"): (1982593280, 259297792),
+    ("c5", "cyclic", "mirrored"): (2706657792, 523120384),
+    ("c5", "sawtooth", "mirrored"): (2469511936, 523371264),
+    ("c5", "cyclic", "none"): (5360406272, 533639168),
+    ("c5", "sawtooth", "none"): (9153945088, 534020096),
 }
 
 
