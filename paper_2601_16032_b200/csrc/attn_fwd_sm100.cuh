@@ -15,6 +15,9 @@
 //                          the TMEM allocation.
 //   the remaining warp(s)  idle; they complete the warpgroup whose registers go to the softmax threads.
 // With two Q tiles the tensor core works on one tile's products while the other tile's softmax runs.
+// Where tensor memory has room for more S buffers than there are Q tiles (d = 64, or a single Q tile), the buffers
+// are handed round in the order of the products, and S of a tile's next step is computed while the softmax of
+// its present step still runs (Geometry::kEarlyQK).
 // Work items come from Algorithm 2's grid-stride walk or, with a counter in global memory, are claimed
 // dynamically; Algorithm 4's scan direction follows the CTA's own item count either way.
 #pragma once
@@ -62,13 +65,22 @@ constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the
 enum WaitSite {
     kSiteProducerQ = 1, kSiteProducerKV = 2, kSiteMmaQ = 3, kSiteMmaKV = 4, kSiteMmaP = 5,
     kSiteSoftmaxS = 6, kSiteSoftmaxO = 7, kSiteSmemAlignment = 8, kSiteWorkFull = 9, kSiteWorkEmpty = 10,
-    kSiteStageSlot = 11, kSiteStageDone = 12
+    kSiteStageSlot = 11, kSiteStageDone = 12, kSiteMmaSFree = 13, kSiteSoftmaxPvDone = 14, kSiteMmaTurn = 15
 };
 
 struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
     uint64_t kv_full[kMaxStages], kv_empty[kMaxStages];
-    uint64_t s_full[2], p_early[2], p_full[2], o_full[2];
+    // Per Q tile and parity of the tile's product count k (two barriers taken in turn, phase (k >> 1) & 1, so that a
+    // completion is never more than one ahead of the role that waits for it): S_q complete; the early part of P_q,
+    // all of P_q written; the product P_q V complete (O_q up to date).
+    uint64_t s_full[2][2], p_early[2][2], p_full[2][2], pv_done[2][2];
+    // Per S buffer (shared by the tiles when there are more buffers than tiles): the P.V product that read its P has
+    // completed.  Its waiters, the two MMA lanes, take turns in the order of the products (qk_turn), so that each use of
+    // a buffer is waited for after the use before it was.
+    uint64_t s_free[4];
+    uint32_t qk_turn;                             // products whose S = Q K^T has been issued
+    uint64_t o_full[2];
     uint64_t drain[2];
     uint64_t stage_done[2];                 // staged epilogue: the four warps of Q tile q have read their staging buffers out
     uint64_t work_full[2], work_empty[2];  // dynamic schedule: two-slot mailbox of claimed work indices
@@ -108,8 +120,16 @@ struct Geometry {
     static constexpr int kRegsOther = 104;
     static constexpr int kRegsSoftmax = 200;
     static constexpr int kTmemCols = 512;
-    static constexpr int kTmemS = 0;      // S_q (fp32, kBlockN columns) at kTmemS + 128 q; P_q aliases its first kBlockN/2 columns
-    static constexpr int kTmemO = 256;    // O_q (fp32, kD columns) at kTmemO + 128 q
+    // Tensor memory: O_q (fp32, kD columns) at kTmemO + kD q, at the top; below it kSBufs buffers of kBlockN columns
+    // for S (fp32), buffer b at kTmemS + kBlockN b; the P of a product overwrites the first half of its S buffer.
+    static constexpr int kTmemO = kTmemCols - kQTiles * kD;
+    static constexpr int kTmemS = 0;
+    static constexpr int kSBufs = kTmemO / kBlockN < 4 ? kTmemO / kBlockN : 4;
+    // As many buffers as tiles: buffer q belongs to tile q, and S_q of the next step can only follow P_q V of this
+    // one.  More buffers than tiles: product n (counted over both tiles, in the order (step, tile)) uses buffer
+    // n mod kSBufs, and a tile's next S product is issued before the MMA lane waits for the tile's present P.
+    static constexpr bool kEarlyQK = kSBufs > kQTiles;
+    static_assert(kSBufs >= kQTiles, "one S buffer per Q tile at least");
     static constexpr size_t smem_bytes(int stages) {
         return (size_t)kQTiles * kQTileBytes + (size_t)stages * kKVTileBytes + sizeof(Barriers);
     }
@@ -166,12 +186,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ptx::mbar_init(&bar->kv_full[s], 1);
             ptx::mbar_init(&bar->kv_empty[s], kQTiles);
         }
+        for (int b = 0; b < 4; ++b) ptx::mbar_init(&bar->s_free[b], 1);
         for (int q = 0; q < 2; ++q) {
-            ptx::mbar_init(&bar->s_full[q], 1);
-            ptx::mbar_init(&bar->p_early[q], 4);   // one arrival per softmax warp of the tile
-            ptx::mbar_init(&bar->p_full[q], 4);
             ptx::mbar_init(&bar->o_full[q], 1);
+            for (int e = 0; e < 2; ++e) {
+                ptx::mbar_init(&bar->s_full[q][e], 1);
+                ptx::mbar_init(&bar->p_early[q][e], 4);   // one arrival per softmax warp of the tile
+                ptx::mbar_init(&bar->p_full[q][e], 4);
+                ptx::mbar_init(&bar->pv_done[q][e], 1);
+            }
         }
+        bar->qk_turn = 0;
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&bar->work_full[i], 1);
             ptx::mbar_init(&bar->work_empty[i], kQTiles + G::kSoftmaxWarps);
@@ -241,6 +266,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         return k;
     };
+
+    // Which S buffer a product uses, and how often that buffer was used before.  idx: products of all tiles before it,
+    // in the order (item, step, tile); every role counts them the same way.
+    struct Product { uint32_t idx; int buf; uint32_t use; };
+    auto product_of = [&](int q, uint32_t idx) -> Product {
+        if (G::kEarlyQK) return Product{idx, (int)(idx % (uint32_t)G::kSBufs), idx / (uint32_t)G::kSBufs};
+        return Product{idx, q, 0u};
+    };
+    // Does Q tile qq of the item take part in step s (its K/V tile lies below the tile's diagonal, and the tile below N)?
+    auto visits = [&](const WorkItem& w, int s, int qq) -> bool { return kv_tile_at(w, s) < (qq ? w.hi_q[1] : w.hi_q[0]); };
 
     if (warp >= G::kSoftmaxWarps) {
     // The last warpgroup (producer, MMA and idle warps) hands registers back in one instruction.  (Its three
@@ -343,16 +378,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t q_base = ptx::smem_u32(q_smem);
         const uint32_t kv_base = ptx::smem_u32(kv_smem);
         Ring ring;
-        uint32_t p_phase = 0;
+        uint32_t n_all = 0, k_mine = 0;   // products so far: of all tiles, of this lane's tile
         bool ok = true;
 
         // Descriptors differ from a base only in the 16-byte-granular address field (the low bits).
         const uint64_t q_desc = ptx::smem_desc_sw128(q_base, 16, 1024) + (uint64_t)((q * G::kQTileBytes) >> 4);
         const uint64_t k_desc0 = ptx::smem_desc_sw128(kv_base, 16, 1024);
         const uint64_t v_desc0 = ptx::smem_desc_sw128(kv_base, G::kKVChunkBytes, 1024);
-        const uint32_t s_tmem = tmem + G::kTmemS + 128 * q;
-        const uint32_t o_tmem = tmem + G::kTmemO + 128 * q;
-        auto issue_qk = [&](int slot) {
+        const uint32_t o_tmem = tmem + G::kTmemO + kD * q;
+        auto issue_qk = [&](int slot, int buf) {
+            const uint32_t s_tmem = tmem + G::kTmemS + kBlockN * buf;
             const uint64_t b0 = k_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
 #pragma unroll
             for (int i = 0; i < G::kChunks * 4; ++i) {
@@ -363,7 +398,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         };
         // The K steps of O_q += P_q V_j whose 16 probabilities belong to the early part of P (late = 0) or
         // to the rest (late = 1); a sum, so the order of the steps is free.
-        auto issue_pv = [&](int slot, uint32_t accumulate, int late) {
+        auto issue_pv = [&](int slot, int buf, uint32_t accumulate, int late) {
+            const uint32_t s_tmem = tmem + G::kTmemS + kBlockN * buf;
             const uint64_t b0 = v_desc0 + (uint64_t)((slot * G::kKVTileBytes) >> 4);
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk) {
@@ -371,6 +407,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ptx::mma_ts(o_tmem, s_tmem + kk * 8, b0 + (uint64_t)(kk * ((16 * 128) >> 4)), idesc_pv,
                             accumulate | (late != 0) | (kk != 0));
             }
+        };
+
+        // More S buffers than tiles: before S of a product goes into a buffer, the products before it have had their S
+        // issued (the lanes take turns), and the P.V product that used the buffer last has completed.
+        auto buffer_free = [&](const Product& pr) -> bool {
+            if (!ptx::spin_until_equal(&bar->qk_turn, pr.idx, abort_flag, kSiteMmaTurn)) return false;
+            return pr.use == 0 || ptx::mbar_wait(&bar->s_free[pr.buf], (pr.use - 1) & 1u, abort_flag, kSiteMmaSFree);
         };
 
         // The elected lane runs the whole loop: every wait, issue and commit below is a single
@@ -396,52 +439,98 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int slot_k = ring.slot;
                 if (!ptx::mbar_wait(&bar->kv_full[slot_k], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
                 ring.advance(stages);
-                ptx::tc_fence_after();
-                if (kv_tile_at(w, 0) < hi_mine) { issue_qk(slot_k); ptx::mma_commit(&bar->s_full[q]); }
+                if (visits(w, 0, q)) {
+                    const Product first = product_of(q, n_all + ((q == 1 && visits(w, 0, 0)) ? 1u : 0u));
+                    if (G::kEarlyQK && !buffer_free(first)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    issue_qk(slot_k, first.buf);
+                    ptx::mma_commit(&bar->s_full[q][k_mine & 1u]);
+                    if (G::kEarlyQK) ptx::st_release_cta(&bar->qk_turn, first.idx + 1);
+                }
                 ptx::mma_commit(&bar->kv_empty[slot_k]);
                 if (w.hi == 1) ptx::mma_commit(&bar->q_empty);
                 uint32_t pv_started = 0;
                 for (int s = 0; ok && s < w.hi; ++s) {
-                    const int j = kv_tile_at(w, s);
                     const bool has_next = s + 1 < w.hi;
-                    const int j_next = has_next ? kv_tile_at(w, s + 1) : 0;
+                    const bool mine = visits(w, s, q);
+                    const bool mine_next = has_next && visits(w, s + 1, q);
+                    const uint32_t in_step = (uint32_t)visits(w, s, 0) + (kQTiles == 2 ? (uint32_t)visits(w, s, 1) : 0u);
+                    const Product cur = product_of(q, n_all + ((q == 1 && visits(w, s, 0)) ? 1u : 0u));
+                    const Product nxt = product_of(q, n_all + in_step + ((q == 1 && has_next && visits(w, s + 1, 0)) ? 1u : 0u));
+                    const uint32_t k_next = k_mine + (mine ? 1u : 0u);   // the tile's product count at its next product
+                    const uint32_t e_cur = k_mine & 1u, ph_cur = (k_mine >> 1) & 1u;
                     const int slot_v = ring.slot;
-                    SAW_PROF(0);
-                    if (!ptx::mbar_wait(&bar->kv_full[slot_v], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                    const uint32_t phase_v = ring.phase;
                     ring.advance(stages);
                     int slot_kn = 0;
-                    if (has_next) {
-                        slot_kn = ring.slot;
-                        if (!ptx::mbar_wait(&bar->kv_full[slot_kn], ring.phase, abort_flag, kSiteMmaKV)) { ok = false; break; }
-                        ring.advance(stages);
+                    uint32_t phase_kn = 0;
+                    if (has_next) { slot_kn = ring.slot; phase_kn = ring.phase; ring.advance(stages); }
+                    SAW_PROF(0);
+                    if (G::kEarlyQK) {
+                        // S of the tile's next step first, into a buffer whose last P has been read; then P.V of this step.
+                        if (has_next) {
+                            if (!ptx::mbar_wait(&bar->kv_full[slot_kn], phase_kn, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                            if (mine_next) {
+                                if (!buffer_free(nxt)) { ok = false; break; }
+                                ptx::tc_fence_after();
+                                issue_qk(slot_kn, nxt.buf);
+                                ptx::mma_commit(&bar->s_full[q][k_next & 1u]);
+                                ptx::st_release_cta(&bar->qk_turn, nxt.idx + 1);
+                                SAW_PROF(7);
+                            }
+                            ptx::mma_commit(&bar->kv_empty[slot_kn]);
+                            if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S product is issued
+                        }
+                        if (!ptx::mbar_wait(&bar->kv_full[slot_v], phase_v, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                        SAW_PROF(2);
+                        if (mine) {
+                            if (!ptx::mbar_wait(&bar->p_early[q][e_cur], ph_cur, abort_flag, kSiteMmaP)) { ok = false; break; }
+                            SAW_PROF(3);
+                            ptx::tc_fence_after();
+                            issue_pv(slot_v, cur.buf, pv_started, 0);
+                            SAW_PROF(4);
+                            if (!ptx::mbar_wait(&bar->p_full[q][e_cur], ph_cur, abort_flag, kSiteMmaP)) { ok = false; break; }
+                            SAW_PROF(5);
+                            ptx::tc_fence_after();
+                            issue_pv(slot_v, cur.buf, pv_started, 1);
+                            pv_started = 1;
+                            ptx::mma_commit(&bar->s_free[cur.buf]);
+                            ptx::mma_commit(&bar->pv_done[q][e_cur]);
+                            SAW_PROF(6);
+                        }
+                        ptx::mma_commit(&bar->kv_empty[slot_v]);
+                    } else {
+                        if (!ptx::mbar_wait(&bar->kv_full[slot_v], phase_v, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                        if (has_next && !ptx::mbar_wait(&bar->kv_full[slot_kn], phase_kn, abort_flag, kSiteMmaKV)) { ok = false; break; }
+                        SAW_PROF(2);
+                        if (mine) {
+                            if (!ptx::mbar_wait(&bar->p_early[q][e_cur], ph_cur, abort_flag, kSiteMmaP)) { ok = false; break; }
+                            SAW_PROF(3);
+                            ptx::tc_fence_after();
+                            issue_pv(slot_v, cur.buf, pv_started, 0);
+                            SAW_PROF(4);
+                            if (!ptx::mbar_wait(&bar->p_full[q][e_cur], ph_cur, abort_flag, kSiteMmaP)) { ok = false; break; }
+                            SAW_PROF(5);
+                            ptx::tc_fence_after();
+                            issue_pv(slot_v, cur.buf, pv_started, 1);
+                            pv_started = 1;
+                            SAW_PROF(6);
+                        }
+                        if (mine_next) {
+                            ptx::tc_fence_after();
+                            issue_qk(slot_kn, nxt.buf);
+                            ptx::mma_commit(&bar->s_full[q][k_next & 1u]);
+                            SAW_PROF(7);
+                        }
+                        // Every lane commits every slot, used by its tile or not: the slot's count is the number of lanes.
+                        ptx::mma_commit(&bar->kv_empty[slot_v]);
+                        if (has_next) {
+                            ptx::mma_commit(&bar->kv_empty[slot_kn]);
+                            if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S product is issued
+                        }
                     }
-                    SAW_PROF(2);
-                    if (j < hi_mine) {
-                        if (!ptx::mbar_wait(&bar->p_early[q], p_phase, abort_flag, kSiteMmaP)) { ok = false; break; }
-                        SAW_PROF(3);
-                        ptx::tc_fence_after();
-                        issue_pv(slot_v, pv_started, 0);
-                        SAW_PROF(4);
-                        if (!ptx::mbar_wait(&bar->p_full[q], p_phase, abort_flag, kSiteMmaP)) { ok = false; break; }
-                        SAW_PROF(5);
-                        p_phase ^= 1u;
-                        ptx::tc_fence_after();
-                        issue_pv(slot_v, pv_started, 1);
-                        pv_started = 1;
-                        SAW_PROF(6);
-                    }
-                    if (has_next && j_next < hi_mine) {
-                        ptx::tc_fence_after();
-                        issue_qk(slot_kn);
-                        ptx::mma_commit(&bar->s_full[q]);
-                        SAW_PROF(7);
-                    }
-                    // Every lane commits every slot, used by its tile or not: the slot's count is the number of lanes.
-                    ptx::mma_commit(&bar->kv_empty[slot_v]);
-                    if (has_next) {
-                        ptx::mma_commit(&bar->kv_empty[slot_kn]);
-                        if (s + 2 == w.hi) ptx::mma_commit(&bar->q_empty);  // the item's last S product is issued
-                    }
+                    n_all += in_step;
+                    k_mine += mine ? 1u : 0u;
                     SAW_PROF(8);
                 }
                 if (!ok) break;
@@ -466,12 +555,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int q = warp >> 2;                       // which Q tile this thread works on
         const int r_in_tile = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + G::kTmemS + 128 * q;
-        const uint32_t t_p = t_s;                      // P overwrites the first half of the row's S columns
-        const uint32_t t_o = tmem + lane_base + G::kTmemO + 128 * q;
+        const uint32_t t_o = tmem + lane_base + G::kTmemO + kD * q;
         const float scale_log2 = p.scale_log2;
         const int N = p.sched.N;
-        uint32_t s_phase = 0, o_phase = 0;
+        uint32_t o_phase = 0;
+        uint32_t n_all = 0, k_mine = 0;   // products so far: of all tiles, of this thread's tile
         bool ok = true;
         int it = 0, slot = 0;
         Ring ring;                 // position of the next work item's first K tile in the K/V ring
@@ -490,7 +578,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ring.advance_by(2 * w.hi, stages);   // now at the item's staging slot
             const Ring stage = ring;
             ring.advance(stages);
-            if (hi_mine == 0) continue;
+            if (hi_mine == 0) {   // the tile lies beyond N: only the other tile's products count
+                n_all += (uint32_t)(w.hi_q[0] + w.hi_q[1]);
+                continue;
+            }
             const int tile_row0 = w.row0 + q * kBlockM;
             const int row = tile_row0 + r_in_tile;
             float m_ref = -INFINITY;   // the max the exponents are taken against (log2 units)
@@ -498,10 +589,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool first = true;
             for (int s = 0; s < w.hi; ++s) {
                 const int j = kv_tile_at(w, s);
-                if (j >= hi_mine) continue;
+                const uint32_t in_step = (uint32_t)visits(w, s, 0) + (kQTiles == 2 ? (uint32_t)visits(w, s, 1) : 0u);
+                if (j >= hi_mine) { n_all += in_step; continue; }
+                const Product cur = product_of(q, n_all + ((q == 1 && visits(w, s, 0)) ? 1u : 0u));
+                const uint32_t e_cur = k_mine & 1u, ph_cur = (k_mine >> 1) & 1u;
+                n_all += in_step;
+                const uint32_t t_s = tmem + lane_base + G::kTmemS + kBlockN * cur.buf;
+                const uint32_t t_p = t_s;              // P overwrites the first half of the row's S columns
                 SAW_PROF(0);
-                const bool got_s = ptx::mbar_wait(&bar->s_full[q], s_phase, abort_flag, kSiteSoftmaxS);
-                s_phase ^= 1u;
+                const bool got_s = ptx::mbar_wait(&bar->s_full[q][e_cur], ph_cur, abort_flag, kSiteSoftmaxS);
                 ptx::tc_fence_after();
                 SAW_PROF(1);
 
@@ -554,7 +650,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         l *= alpha;
                     }
                     if (!first) {
-                        // S_q is complete, so every product issued before it, O_q's last update included, is too.
+                        // O_q's last update must have completed.  It was issued before this S product, which is
+                        // complete, unless S products run ahead: then the update has a barrier of its own.
+                        if (G::kEarlyQK) {
+                            ok = ptx::warp_all(ptx::mbar_wait(&bar->pv_done[q][(k_mine - 1) & 1u], ((k_mine - 1) >> 1) & 1u, abort_flag,
+                                                              kSiteSoftmaxPvDone));
+                            if (!ok) break;
+                            ptx::tc_fence_after();
+                        }
 #pragma unroll 1
                         for (int c = 0; c < kColsO / 16; ++c) {
                             uint32_t ov[16];
@@ -581,7 +684,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         ptx::tmem_wait_st();
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bar->p_early[q]);
+                        if (lane == 0) ptx::mbar_arrive(&bar->p_early[q][e_cur]);
                         SAW_PROF(6);
                     }
                 };
@@ -616,9 +719,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&bar->p_full[q]);
+                if (lane == 0) ptx::mbar_arrive(&bar->p_full[q][e_cur]);
                 SAW_PROF(7);
                 first = false;
+                ++k_mine;
             }
             if (!ok) break;
             // ---- epilogue: O_q / l -> 16 bit -> global

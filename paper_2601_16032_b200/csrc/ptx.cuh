@@ -84,6 +84,27 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return mbar_wait_slow(bar, parity, abort_flag, where);
 }
 
+// A word in shared memory that one thread of the CTA writes (release) and another polls (acquire).
+__device__ __forceinline__ void st_release_cta(uint32_t* addr, uint32_t v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(addr)), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_cta(const uint32_t* addr) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(addr)) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool spin_until_equal(const uint32_t* addr, uint32_t want, volatile int* abort_flag, int where) {
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (ld_acquire_cta(addr) == want) return true;
+        if (*abort_flag != 0) return false;
+        if (global_ns() - t0 > kWaitBudgetNs) break;
+    }
+    if (*abort_flag == 0) *abort_flag = where;
+    return false;
+}
+
 // ---------------------------------------------------------------- TMA (tiled bulk tensor copies)
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -65,6 +65,9 @@ CONFIGS = {
 STUDY_CASES = {
     "c3-small": Workload("c3-small", 2, 16, 8192, 128, BF16, False, 2003),
     "c4-small": Workload("c4-small", 1, 8, 32768, 128, BF16, True, 2004, k_scale=0.5),
+    # The paper's head dimension at a size that fills the GPU several times over, and a capture-sized half of it.
+    "d64-n8k": Workload("d64-n8k", 4, 16, 8192, 64, F16, False, 2064),
+    "d64-n8k-small": Workload("d64-n8k-small", 2, 16, 8192, 64, F16, False, 2065),
     "long-64k": Workload("long-64k", 1, 1, 65536, 128, BF16, False, 2010),
     "long-128k": Workload("long-128k", 1, 1, 131072, 128, BF16, False, 2011),
     "long-192k": Workload("long-192k", 1, 1, 196608, 128, BF16, False, 2012),
