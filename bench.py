@@ -4,7 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--also c3,c4] [--impl reference]
 
 Prints ONE JSON line.  The workload is c5 (B=2 H=16 N=65536 d=128 bf16 causal), the largest of the five
-configurations; c3 and c4 are measured the same way and reported, each with its own roofline block, under `also`.
+configurations; c3, c4, c2 and a d = 64 shape that fills the GPU (d64-n8k) are measured the same way and reported, each
+with its own roofline block, under `also`.
 
 How a workload is timed.  The two scan orders are launched in alternation, cyclic, sawtooth, cyclic, ..., every
 launch between its own pair of CUDA events on the launch stream, after a warm-up of the same alternating launches
@@ -365,6 +366,14 @@ class Bench:
                          "dram_read_bytes": dram[0] if dram else None, "compulsory_read_bytes": 3 * w.compulsory_bytes // 4,
                          "read_amplification": (dram[0] / (3 * w.compulsory_bytes / 4)) if dram else None},
         }
+        if w.d == 64:
+            # The tensor work of a step halves at d = 64 and its softmax does not: the step is as long as the softmax of a
+            # tile, which is bound by the schedulers' issue slots and the MUFU.  Counters of one launch (ncu, d64-n8k-small):
+            # 1466 instructions issued per scheduler and step, 1536 MUFU cycles per scheduler and step.
+            cps = legs[headline]["cycles_per_kv_step"]
+            block["roofline"]["alu"] = {"bound": "alu", "what": "softmax of two Q tiles per K/V step on each of the SM's four schedulers",
+                                        "issue_slots_per_step": 1466, "mufu_cycles_per_step": 1536,
+                                        "frac_issue": 1466 / cps, "frac_mufu": 1536 / cps}
         if len(seq) == 2:
             block["sawtooth_over_cyclic"] = float(np.mean(per_order["cyclic"]) / np.mean(per_order["sawtooth"]))
         return block, devb, launch
@@ -425,7 +434,7 @@ def main():
     ap.add_argument("--pairing", default="default", choices=["default", "none", "mirrored", "adjacent"],
                     help="how the static walk groups work items (default: mirrored pairs under the causal mask)")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the persistent grid (the paper's 'active SMs'); 0 = all SMs")
-    ap.add_argument("--also", default="c3,c4",
+    ap.add_argument("--also", default="c3,c4,d64-n8k,c2",
                     help="further workloads measured the same way (single GPU only; '' for none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (default: min(steps, 5))")
