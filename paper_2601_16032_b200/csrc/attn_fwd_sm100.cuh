@@ -55,10 +55,15 @@ struct KernelParams {
 };
 
 constexpr int kMaxStages = 16;
-#ifndef SAW_EXP_POLY_OF_4
-#define SAW_EXP_POLY_OF_4 1
+// Which of the eight pairs of exponentials of a group of 16 avoid the MUFU (bit i: pair i takes the cubic on the FMA
+// pipe).  At d = 64 the step is as long as the softmax and a quarter of them off the MUFU is the measured optimum; at
+// d = 128 the tensor core sets the step, the MUFU has room, and the extra instructions only cost power.
+#ifndef SAW_EXP_POLY_MASK_D64
+#define SAW_EXP_POLY_MASK_D64 0x11
 #endif
-constexpr int kExpPolyOf4 = SAW_EXP_POLY_OF_4;  // of every four pairs of exponentials, how many avoid the MUFU
+#ifndef SAW_EXP_POLY_MASK_D128
+#define SAW_EXP_POLY_MASK_D128 0x00
+#endif
 constexpr float kRescaleThreshold = 8.0f;  // O and l are rescaled only when the row max grew by more (log2 units)
 
 // Codes written to the status word: which wait gave up.
@@ -552,6 +557,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // ------------------------------------------------------------------ softmax / correction / epilogue
         if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
         constexpr int kColsS = G::kColsS, kColsO = G::kColsO;
+        constexpr int kExpPolyMask = kD == 64 ? SAW_EXP_POLY_MASK_D64 : SAW_EXP_POLY_MASK_D128;
         const int q = warp >> 2;                       // which Q tile this thread works on
         const int r_in_tile = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -694,15 +700,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 16; i += 4) {
                         // Four probabilities: x = S * scale * log2(e) - m as two packed FMAs, then 2^x on the MUFU
-                        // or, for kExpPolyOf4 of every four pairs, on the FMA pipe.
+                        // or, for the pairs of the group that kExpPolyMask names, on the FMA pipe.
                         const ptx::f32x2 xa = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i]), __uint_as_float(sv[c][16 * h + i + 1])), scale2, neg_m2);
                         const ptx::f32x2 xb = ptx::fma2(ptx::pack_f32x2(__uint_as_float(sv[c][16 * h + i + 2]), __uint_as_float(sv[c][16 * h + i + 3])), scale2, neg_m2);
                         float x0, x1, x2, x3, p0, p1, p2, p3;
                         ptx::unpack_f32x2(xa, x0, x1);
                         ptx::unpack_f32x2(xb, x2, x3);
-                        if (((i >> 2) * 2) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x0, x1, p0, p1);
+                        if ((kExpPolyMask >> ((i >> 2) * 2)) & 1) ptx::exp2_poly_pair(x0, x1, p0, p1);
                         else { p0 = ptx::ex2(x0); p1 = ptx::ex2(x1); }
-                        if (((i >> 2) * 2 + 1) % 4 < kExpPolyOf4) ptx::exp2_poly_pair(x2, x3, p2, p3);
+                        if ((kExpPolyMask >> ((i >> 2) * 2 + 1)) & 1) ptx::exp2_poly_pair(x2, x3, p2, p3);
                         else { p2 = ptx::ex2(x2); p3 = ptx::ex2(x3); }
                         l01 = ptx::add2(l01, ptx::pack_f32x2(p0, p1));
                         l23 = ptx::add2(l23, ptx::pack_f32x2(p2, p3));
