@@ -66,6 +66,64 @@ __global__ void __launch_bounds__(kThreads, 1) mma_rate(int n_cols, int a_in_tme
     if (warp == 0) { ptx::tc_fence_after(); ptx::tmem_dealloc(tmem, 512); }
 }
 
+// The same measurement with the shared-memory operands in the other K-major layouts the descriptor knows: rows of 64
+// bytes (64-byte swizzle), rows of 32 bytes (32-byte swizzle: one row is exactly one K step) and unswizzled 8 x 16-byte
+// core matrices.  layout: 0 = 128-byte swizzle, 1 = 64-byte, 2 = 32-byte, 3 = none.  One issuing thread, N = 128.
+__device__ __forceinline__ uint64_t desc_for_step(uint32_t base, int layout, int i) {
+    // address of K step i (16 elements, 32 bytes of every row) of a 128-row operand, and the strides of its layout
+    uint32_t addr, lbo, sbo;
+    uint64_t swizzle;
+    if (layout == 0) { addr = base + (i >> 2) * 16384 + (i & 3) * 32; lbo = 16; sbo = 1024; swizzle = 2; }
+    else if (layout == 1) { addr = base + (i >> 1) * 8192 + (i & 1) * 32; lbo = 16; sbo = 512; swizzle = 4; }
+    else if (layout == 2) { addr = base + i * 4096; lbo = 16; sbo = 256; swizzle = 6; }
+    else { addr = base + i * 4096; lbo = 128; sbo = 256; swizzle = 0; }
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= swizzle << 61;
+    return d;
+}
+__global__ void __launch_bounds__(kThreads, 1) mma_rate_layout(int a_layout, int b_layout, int a_in_tmem, int batches, unsigned long long* out, int* status) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t done;
+    __shared__ uint32_t tmem_base;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < kSmemBytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) { ptx::mbar_init(&done, 1); abort_flag = 0; ptx::fence_mbar_init(); }
+    ptx::fence_proxy_async_smem();
+    if (warp == 0) { ptx::tmem_alloc(&tmem_base, 512); ptx::tmem_relinquish(); }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = tmem_base;
+    if (warp == 1 && ptx::elect_one()) {
+        const uint32_t base = ptx::smem_u32(smem);
+        uint64_t ad[8], bd[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { ad[i] = desc_for_step(base, a_layout, i); bd[i] = desc_for_step(base + 32768, b_layout, i); }
+        const uint32_t idesc = ptx::instr_desc_f16(1, 0, 128, 128);
+        const long long t0 = clock64();
+        for (int it = 0; it < batches; ++it) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (a_in_tmem) ptx::mma_ts(tmem, tmem + 128 + i * 8, bd[i], idesc, 1);
+                else ptx::mma_ss(tmem, ad[i], bd[i], idesc, 1);
+            }
+        }
+        ptx::mma_commit(&done);
+        const bool ok = ptx::mbar_wait(&done, 0, &abort_flag, 1);
+        const long long t1 = clock64();
+        if (blockIdx.x == 0) out[0] = (unsigned long long)(t1 - t0);
+        if (!ok) atomicExch(status, 1);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) { ptx::tc_fence_after(); ptx::tmem_dealloc(tmem, 512); }
+}
+
 // The same measurement for the two-SM form (cta_group::2): a cluster of two CTAs, M = 256 (128 rows in each CTA's tensor
 // memory), N = 128 with each CTA holding 64 of the 128 B rows in its own shared memory; one thread of the cluster's first
 // CTA issues for both.
@@ -161,6 +219,24 @@ int main() {
                 const char* where[4] = {"smem", "TMEM", "smem and TMEM alternating in each thread", "smem (even threads) / TMEM (odd threads)"};
                 printf("A in %s, N = %3d, %d issuing thread(s): %6.1f cycles per MMA, %5.0f FLOP/clk/SM (status %d)\n",
                        where[a_in_tmem], n, issuers, per, 2.0 * 128 * n * 16 / per, st);
+            }
+    cudaFuncSetAttribute(mma_rate_layout, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    const char* layout_name[4] = {"128-byte swizzle", "64-byte swizzle", "32-byte swizzle", "no swizzle"};
+    for (int a_in_tmem = 0; a_in_tmem < 2; ++a_in_tmem)
+        for (int a_layout = 0; a_layout < (a_in_tmem ? 1 : 4); ++a_layout)
+            for (int b_layout = 0; b_layout < 4; ++b_layout) {
+                for (int rep = 0; rep < 2; ++rep) {
+                    mma_rate_layout<<<sms, kThreads, kSmemBytes>>>(a_layout, b_layout, a_in_tmem, batches, out, status);
+                    cudaError_t e = cudaDeviceSynchronize();
+                    if (e != cudaSuccess) { printf("error %s\n", cudaGetErrorString(e)); return 1; }
+                }
+                unsigned long long cycles = 0;
+                int st = 0;
+                cudaMemcpy(&cycles, out, 8, cudaMemcpyDeviceToHost);
+                cudaMemcpy(&st, status, 4, cudaMemcpyDeviceToHost);
+                const double per = (double)cycles / (8.0 * batches);
+                printf("layouts: A %s, B K-major %s, N = 128, 1 issuing thread: %6.1f cycles per MMA (status %d)\n",
+                       a_in_tmem ? "in TMEM" : layout_name[a_layout], layout_name[b_layout], per, st);
             }
     cudaFuncSetAttribute(mma_rate_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     for (int a_in_tmem = 0; a_in_tmem < 2; ++a_in_tmem) {
