@@ -79,7 +79,7 @@ typedef struct {
     int digit_order;  /* attn_digit_order: how the linear work index maps to (batch, head, Q block) */
     int launch_mode;  /* 0: persistent grid (Algorithm 2); 1: one CTA per work item (Algorithm 3) */
     int l2_policy;    /* 0: no hint; 1: K/V loads carry an evict_last hint, Q loads evict_first */
-    int host_chunks;  /* attn_fwd_host only: pieces the heads are cut into so that copies and kernels overlap (1..16; 0 = automatic) */
+    int host_chunks;  /* attn_fwd_host only: pieces the heads are cut into so that copies and kernels overlap (1..32; 0 = automatic) */
     float* lse;       /* optional DEVICE output [B, H, N] (fp32, 4-byte aligned), NULL for none: per query row the natural log of
                          the softmax denominator, ln sum_j exp(scale * q_i . k_j) over the keys the row may see (the quantity a
                          backward pass or a merge of partial results needs; outside the paper).  Ignored by attn_fwd_host. */
@@ -185,8 +185,12 @@ int attn_fwd_dynamic_noalloc(const void* q, const void* k, const void* v, void* 
  * Same computation for HOST buffers: copies q, k, v (host, pinned if the copies are to overlap anything) into the
  * caller's device staging buffers q_dev, k_dev, v_dev, runs attn_fwd_ex into o_dev and copies o_dev back to o_host.
  * Each buffer holds B*H*N*d 16-bit elements.  The heads are independent, so the work is cut into opts->host_chunks
- * groups of heads (automatic: up to 8 once a tensor exceeds 32 MiB) that run as a pipeline on three streams the
- * library keeps per device: upload of group i+1, kernel of group i and download of group i-1 proceed together.  The
+ * equal groups of heads; left to the library (0), one group per 16 MiB of a tensor once a tensor exceeds 32 MiB, 32
+ * at most and a head at least (attn_host_groups tells which): upload and kernel take about as long as each other on a
+ * PCIe 5 link, so the first kernel should start early and none should wait for a long upload.  The groups run as a
+ * pipeline on streams the library keeps per device: upload of group i+1, kernel of group i and download of group i-1
+ * proceed together, and the kernels of successive groups alternate between two streams, so that the CTAs of group i+1
+ * move onto the SMs that the last round of group i leaves idle.  The
  * pipeline starts after everything already enqueued on `stream` and `stream` waits for its end, so to the caller it
  * behaves like work enqueued on `stream`.  Returns without waiting: o_host is valid once `stream` has been
  * synchronised.  The first pipelined call on a device creates the streams and events (no device memory).
@@ -199,6 +203,13 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
                   void* q_dev, void* k_dev, void* v_dev, void* o_dev,
                   int B, int H, int N, int d, float scale, int causal, int scan_order,
                   int dtype, void* stream, const attn_fwd_opts* opts);
+
+/*
+ * Host-only: the groups of heads attn_fwd_host cuts B*H = `heads` heads of `head_bytes` bytes each into, for
+ * opts->host_chunks = host_chunks.  Writes the group sizes, in order, to sizes[0 .. *n - 1]; `sizes` holds at least 32
+ * entries.  They sum to `heads`.  The paper has no counterpart: it times kernels on resident tensors.
+ */
+int attn_host_groups(long long heads, size_t head_bytes, int host_chunks, long long* sizes, int* n);
 
 /*
  * The launch plan for these arguments (Algorithm 2's grid size, the tile shapes).  sm_count <= 0

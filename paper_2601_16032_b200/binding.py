@@ -76,6 +76,8 @@ def load_library():
     lib.attn_query_plan.argtypes = shape + [ci, ci, ctypes.POINTER(Opts), ci, ctypes.POINTER(Plan)]
     lib.attn_schedule_trace.argtypes = shape + [ci, ci, ci, ctypes.POINTER(Opts), ci, ctypes.POINTER(TraceEntry),
                                                 ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+    lib.attn_host_groups.argtypes = [ctypes.c_longlong, ctypes.c_size_t, ci, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ci)]
+    lib.attn_host_groups.restype = ci
     lib.attn_device_status.argtypes = [ctypes.POINTER(ci)]
     lib.attn_last_kernel_cycles.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
     lib.attn_last_kernel_cycles.restype = ci
@@ -160,6 +162,14 @@ def attn_schedule_trace(B: int, H: int, N: int, d: int, causal: int, scan_order:
     buf = (TraceEntry * n.value)()
     _check(lib.attn_schedule_trace(B, H, N, d, int(causal), scan_order, dtype, _opts_ptr(opts), sm_count, buf, n.value, ctypes.byref(n)))
     return list(buf)
+
+
+def attn_host_groups(heads: int, head_bytes: int, host_chunks: int = 0) -> list:
+    """The groups of heads attn_fwd_host cuts its work into (host-only)."""
+    sizes = (ctypes.c_longlong * 32)()
+    n = ctypes.c_int(0)
+    _check(load_library().attn_host_groups(ctypes.c_longlong(heads), ctypes.c_size_t(head_bytes), host_chunks, sizes, ctypes.byref(n)))
+    return [int(sizes[i]) for i in range(n.value)]
 
 
 def attn_device_status() -> int:

@@ -33,7 +33,7 @@ __device__ unsigned long long g_cycles = 0;
 static __device__ __align__(256) int g_noalloc_scratch[(ATTN_DYNAMIC_SCRATCH_HEADER / 4) + ATTN_NOALLOC_MAX_CTAS];
 
 constexpr int kMaxDevices = 64;
-constexpr int kMaxHostChunks = 16;
+constexpr int kMaxHostChunks = 32;
 constexpr int kSmemOptinB200 = 232448;  // 227 KiB of dynamic shared memory per CTA on sm_100
 constexpr int kKernelVariants = 16;     // d x block_n x q_tiles x dtype
 
@@ -491,8 +491,8 @@ namespace {
 struct HostPipe {
     std::mutex busy;
     bool ready = false;
-    cudaStream_t up = nullptr, run = nullptr, down = nullptr;
-    cudaEvent_t start = nullptr, done_up = nullptr, done_run = nullptr, done_down = nullptr;
+    cudaStream_t up = nullptr, run[2] = {nullptr, nullptr}, down = nullptr;
+    cudaEvent_t start = nullptr, done_up = nullptr, done_run[2] = {nullptr, nullptr}, done_down = nullptr;
     cudaEvent_t uploaded[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {};
 };
 HostPipe g_host_pipe[kMaxDevices];
@@ -501,11 +501,13 @@ HostPipe g_host_pipe[kMaxDevices];
 int prepare_host_pipe(HostPipe& hp) {
     if (hp.ready) return ATTN_OK;
     bool ok = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaStreamCreateWithFlags(&hp.run, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.run[0], cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.run[1], cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) == cudaSuccess &&
               cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
               cudaEventCreateWithFlags(&hp.done_up, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&hp.done_run, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done_run[0], cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done_run[1], cudaEventDisableTiming) == cudaSuccess &&
               cudaEventCreateWithFlags(&hp.done_down, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; ok && i < kMaxHostChunks; ++i)
         ok = cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) == cudaSuccess &&
@@ -514,7 +516,30 @@ int prepare_host_pipe(HostPipe& hp) {
     hp.ready = true;
     return ATTN_OK;
 }
+
+// Groups of heads for attn_fwd_host: host_chunks equal ones (the first ones a head larger when it does not divide), or,
+// left to the library, one group per 16 MiB of a tensor once the tensor exceeds 32 MiB (kMaxHostChunks at most, a head
+// at least).  Small equal groups: upload and kernel take about as long as each other on a PCIe 5 link, so what counts
+// is that the first kernel starts early and that no kernel waits for a long upload.
+int host_groups(long long heads, size_t head_bytes, int host_chunks, long long* group) {
+    long long chunks = host_chunks;
+    if (chunks == 0) {
+        const size_t bytes = (size_t)heads * head_bytes;
+        chunks = bytes > ((size_t)32 << 20) ? (long long)(bytes >> 24) : 1;
+        if (chunks > kMaxHostChunks) chunks = kMaxHostChunks;
+    }
+    if (chunks > heads) chunks = heads;
+    for (long long ch = 0; ch < chunks; ++ch) group[ch] = heads / chunks + (ch < heads % chunks ? 1 : 0);
+    return (int)chunks;
+}
 }  // namespace
+
+int attn_host_groups(long long heads, size_t head_bytes, int host_chunks, long long* sizes, int* n) {
+    if (heads <= 0 || head_bytes == 0 || !sizes || !n) return fail(ATTN_ERR_INVALID_ARG, "heads and head_bytes must be positive, sizes and n non-null");
+    if (host_chunks < 0 || host_chunks > kMaxHostChunks) return fail(ATTN_ERR_INVALID_ARG, "host_chunks must be in [0, %d]", kMaxHostChunks);
+    *n = host_groups(heads, head_bytes, host_chunks, sizes);
+    return ATTN_OK;
+}
 
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, void* q_dev, void* k_dev,
                   void* v_dev, void* o_dev, int B, int H, int N, int d, float scale, int causal, int scan_order, int dtype,
@@ -535,9 +560,8 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
     const long long heads = (long long)B * H;
-    int chunks = inner.host_chunks;
-    if (chunks == 0) chunks = bytes > ((size_t)32 << 20) ? 8 : 1;
-    if (chunks > heads) chunks = (int)heads;
+    long long group[kMaxHostChunks];
+    const int chunks = host_groups(heads, (size_t)N * d * 2, inner.host_chunks, group);
     if (chunks <= 1) {
         if ((e = cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
             (e = cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
@@ -553,7 +577,9 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
         }
         return ATTN_OK;
     }
-    // Pipeline over groups of heads: upload, kernel and download of successive groups overlap on three streams.
+    // Pipeline over groups of heads: upload, kernel and download of successive groups overlap.  The kernels alternate
+    // between two streams: a group's launch rarely fills its last round of work items, and the next group's CTAs move
+    // onto the SMs that fall idle (the two kernels share nothing but read-only options).
     HostPipe& hp = g_host_pipe[c.dev];
     std::lock_guard<std::mutex> lock(hp.busy);
     if ((rc = prepare_host_pipe(hp))) return rc;
@@ -567,11 +593,13 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
         return err == cudaSuccess;
     };
     check(cudaStreamWaitEvent(hp.up, hp.start, 0), "cudaStreamWaitEvent");
-    check(cudaStreamWaitEvent(hp.run, hp.start, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(hp.run[0], hp.start, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(hp.run[1], hp.start, 0), "cudaStreamWaitEvent");
     check(cudaStreamWaitEvent(hp.down, hp.start, 0), "cudaStreamWaitEvent");
     long long h0 = 0;
     for (int ch = 0; ch < chunks && !failed && rc == 0; ++ch) {
-        const long long n_heads = heads / chunks + (ch < heads % chunks ? 1 : 0);
+        const long long n_heads = group[ch];
+        cudaStream_t run = hp.run[ch & 1];
         const size_t off = (size_t)h0 * head_bytes, len = (size_t)n_heads * head_bytes;
         const uint8_t *qh = (const uint8_t*)q_host + off, *kh = (const uint8_t*)k_host + off, *vh = (const uint8_t*)v_host + off;
         uint8_t *qd = (uint8_t*)q_dev + off, *kd = (uint8_t*)k_dev + off, *vd = (uint8_t*)v_dev + off, *od = (uint8_t*)o_dev + off;
@@ -579,11 +607,11 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
             !check(cudaMemcpyAsync(kd, kh, len, cudaMemcpyHostToDevice, hp.up), "host-to-device copy") ||
             !check(cudaMemcpyAsync(vd, vh, len, cudaMemcpyHostToDevice, hp.up), "host-to-device copy") ||
             !check(cudaEventRecord(hp.uploaded[ch], hp.up), "cudaEventRecord") ||
-            !check(cudaStreamWaitEvent(hp.run, hp.uploaded[ch], 0), "cudaStreamWaitEvent"))
+            !check(cudaStreamWaitEvent(run, hp.uploaded[ch], 0), "cudaStreamWaitEvent"))
             break;
-        rc = attn_fwd_ex(qd, kd, vd, od, 1, (int)n_heads, N, d, scale, causal, scan_order, dtype, hp.run, &inner);
+        rc = attn_fwd_ex(qd, kd, vd, od, 1, (int)n_heads, N, d, scale, causal, scan_order, dtype, run, &inner);
         if (rc) break;
-        if (!check(cudaEventRecord(hp.computed[ch], hp.run), "cudaEventRecord") ||
+        if (!check(cudaEventRecord(hp.computed[ch], run), "cudaEventRecord") ||
             !check(cudaStreamWaitEvent(hp.down, hp.computed[ch], 0), "cudaStreamWaitEvent") ||
             !check(cudaMemcpyAsync((uint8_t*)o_host + off, od, len, cudaMemcpyDeviceToHost, hp.down), "device-to-host copy"))
             break;
@@ -591,10 +619,12 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     }
     // Join: `stream` continues only after everything enqueued on the three side streams, on success and on failure alike.
     check(cudaEventRecord(hp.done_up, hp.up), "cudaEventRecord");
-    check(cudaEventRecord(hp.done_run, hp.run), "cudaEventRecord");
+    check(cudaEventRecord(hp.done_run[0], hp.run[0]), "cudaEventRecord");
+    check(cudaEventRecord(hp.done_run[1], hp.run[1]), "cudaEventRecord");
     check(cudaEventRecord(hp.done_down, hp.down), "cudaEventRecord");
     check(cudaStreamWaitEvent(st, hp.done_up, 0), "cudaStreamWaitEvent");
-    check(cudaStreamWaitEvent(st, hp.done_run, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(st, hp.done_run[0], 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(st, hp.done_run[1], 0), "cudaStreamWaitEvent");
     check(cudaStreamWaitEvent(st, hp.done_down, 0), "cudaStreamWaitEvent");
     if (rc) return rc;   // attn_fwd_ex's own message stands
     if (failed) return fail(ATTN_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));

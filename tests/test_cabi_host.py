@@ -140,3 +140,27 @@ def check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits, pair
             else:
                 assert n_q == sch.kv_tiles_needed(r // 128, N, 128, block_n, bool(causal))
         assert max(g.n_kv_q0, g.n_kv_q1) == g.n_kv
+
+
+def test_host_groups():
+    """attn_fwd_host's groups of heads: equal ones on request; left to the library, one group for small tensors and
+    otherwise one per 16 MiB of a tensor, 32 at most, a head at least."""
+    mib = 1 << 20
+    assert sa.attn_host_groups(32, 16 * mib) == [1] * 32                           # c5: 32 heads of 16 MiB
+    assert sa.attn_host_groups(32, 8 * mib) == [2] * 16                            # c4
+    assert sa.attn_host_groups(64, 2 * mib) == [8] * 8                             # c3
+    assert sa.attn_host_groups(5, 64 * mib) == [1] * 5
+    assert sa.attn_host_groups(1, 64 * mib) == [1]
+    assert sa.attn_host_groups(8, 1 * mib) == [8]                                  # 8 MiB: not worth a pipeline
+    assert sa.attn_host_groups(8, 4 * mib) == [8]                                  # 32 MiB: not yet
+    assert sa.attn_host_groups(10, 16 * mib, 3) == [4, 3, 3]
+    assert sa.attn_host_groups(2, 16 * mib, 16) == [1, 1]
+    for heads in list(range(1, 200)) + [1000, 4096, 100000]:
+        for chunks in (0, 1, 7, 32):
+            g = sa.attn_host_groups(heads, 3 * mib, chunks)
+            assert sum(g) == heads and len(g) <= 32 and min(g) >= 1 and max(g) - min(g) <= 1
+            assert g == sorted(g, reverse=True)
+    with pytest.raises(sa.AttnError):
+        sa.attn_host_groups(0, mib)
+    with pytest.raises(sa.AttnError):
+        sa.attn_host_groups(4, mib, 33)

@@ -141,7 +141,7 @@ def test_bad_arguments_are_rejected_before_launch():
         assert e.value.status == status, (change, e.value)
 
 
-@pytest.mark.parametrize("host_chunks", [1, 3, 16])
+@pytest.mark.parametrize("host_chunks", [1, 3, 32])
 def test_host_entry_point_pipeline_matches_device_entry_point(host_chunks):
     """attn_fwd_host (pinned host buffers in and out, heads cut into groups that are uploaded, computed and
     downloaded as a pipeline) gives the device entry point's result bit for bit in the cyclic order."""
@@ -165,6 +165,32 @@ def test_host_entry_point_pipeline_matches_device_entry_point(host_chunks):
         sa.attn_device_status()
         assert torch.equal(o_host, want.view(torch.int16).cpu())
     assert_parity(w, o_host.view(torch.bfloat16).cuda())
+
+
+def test_host_entry_point_with_the_library_own_groups():
+    """A tensor above 32 MiB, host_chunks left at 0: attn_fwd_host cuts the nine heads into two groups and runs their
+    kernels on two streams in turn; the result is the device entry point's up to the scan directions."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("host-ramp", 1, 9, 16384, 128, wl.BF16, True, 7355)
+    assert sa.attn_host_groups(w.B * w.H, w.N * w.d * 2) == [5, 4]
+    q, k, v = upload(w)
+    want = run_cuda(w, (q, k, v), sa.SAWTOOTH)
+    host = [t.view(torch.int16).cpu().pin_memory() for t in (q, k, v)]
+    o_host = torch.full(q.shape, -1, dtype=torch.int16).pin_memory()
+    dev = [torch.empty_like(q) for _ in range(4)]
+    stream = torch.cuda.Stream()
+    for _ in range(2):
+        o_host.fill_(-1)
+        sa.attn_fwd_host(host[0].data_ptr(), host[1].data_ptr(), host[2].data_ptr(), o_host.data_ptr(), dev[0].data_ptr(),
+                         dev[1].data_ptr(), dev[2].data_ptr(), dev[3].data_ptr(), w.B, w.H, w.N, w.d, w.scale, 1, sa.SAWTOOTH,
+                         sa.BF16, stream.cuda_stream, None)
+        stream.synchronize()
+        sa.attn_device_status()
+        # a group is a launch of its own: its heads' items land on other CTAs, with other scan directions, than in one launch
+        got = o_host.view(torch.bfloat16).cuda()
+        assert (got.float() - want.float()).abs().max().item() < 2e-2
+    assert_parity(w, got, {bh: wl.sampled_rows(w, bh[0], bh[1], 48) for bh in wl.all_heads(w)})
 
 
 @pytest.mark.parametrize("causal", [False, True])
