@@ -1,4 +1,4 @@
-"""The cubic the kernel uses for 2^f on the FMA pipe (a quarter of the exponentials): its coefficients are read from
+"""The cubic the kernel uses for 2^f on the FMA pipe (a quarter of the exponentials at d = 64): its coefficients are read from
 the CUDA header and checked on the host against 2^f in fp64, evaluated in fp32 Horner form as the kernel does, and the
 range reduction (floor taken from the low mantissa bits of x + 1.5 * 2^23) is replayed with numpy integers."""
 import os
