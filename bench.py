@@ -420,6 +420,21 @@ class Bench:
         return float(np.median(times))
 
 
+def host_call_us_from_c():
+    """The same call timed from C (profile_host_call.cu, built beside the library): what the library itself costs per
+    call, without the ctypes marshalling.  None when the program is not there and cannot be built."""
+    import re
+    import subprocess
+    try:
+        from paper_2601_16032_b200 import build as lib_build
+        exe = lib_build.build_host_call_probe()
+        out = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+        m = re.search(r"median ([0-9.]+) us", out.stdout)
+        return float(m.group(1)) if out.returncode == 0 and m else None
+    except Exception:
+        return None
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -475,6 +490,7 @@ def main():
     block, devb, launch = bench.measure(w, args.steps, args.warmup, headline, only, host)
     dyn = bench.dynamic_leg(w, devb, launch, headline, max(3, min(args.steps, 10))) if only is None else None
     host_us = bench.host_call_us()
+    host_us_c = host_call_us_from_c() if rank == 0 else None
 
     # End to end: host buffers in, host buffer out, copies inside the timed region.
     e2e = None
@@ -524,7 +540,7 @@ def main():
         "gpu_launches": block["launches_in_timed_region"],
         "roofline": block["roofline"],
         "orders": block["orders"], "single_launch": block["single_launch"], "ms_per_step_median": block["ms_per_step_median"],
-        "host_call_us": host_us,
+        "host_call_us": host_us, "host_call_us_from_c": host_us_c,
     }
     if "sawtooth_over_cyclic" in block:
         line["sawtooth_over_cyclic"] = block["sawtooth_over_cyclic"]

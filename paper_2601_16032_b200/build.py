@@ -36,6 +36,23 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+HOST_CALL_SRC = os.path.join(ROOT, "profile_host_call.cu")
+HOST_CALL_BIN = os.path.join(PKG, "profile_host_call")
+
+
+def build_host_call_probe(force: bool = False) -> str:
+    """Builds the C program that times one attn_fwd call from C (a measuring aid of bench.py) against the in-tree library."""
+    build()
+    if not force and os.path.exists(HOST_CALL_BIN) and os.path.getmtime(HOST_CALL_BIN) >= max(os.path.getmtime(HOST_CALL_SRC), os.path.getmtime(LIB)):
+        return HOST_CALL_BIN
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-O2", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-o", HOST_CALL_BIN, HOST_CALL_SRC,
+           "-L" + PKG, "-lsawtooth_attn", "-Xlinker", "-rpath", "-Xlinker", "$ORIGIN"]
+    subprocess.run(cmd, check=True, cwd=ROOT)
+    return HOST_CALL_BIN
+
+
 if __name__ == "__main__":
     import sys
     print(build(force=True, verbose="-v" in sys.argv))
+    print(build_host_call_probe(force=True))
