@@ -352,6 +352,41 @@ def test_many_one_tile_items_per_cta(N, kv_stages):
         assert torch.equal(o.view(torch.int16), want.view(torch.int16))
 
 
+@pytest.mark.parametrize("shape", [(64, 128, 2), (64, 64, 2), (64, 128, 1), (128, 128, 1), (128, 64, 2), (128, 64, 1)],
+                         ids=lambda t: f"d{t[0]}bn{t[1]}q{t[2]}")
+@pytest.mark.parametrize("N,causal", [(129, False), (257, False), (385, True), (641, True), (900, False)])
+@pytest.mark.parametrize("kv_stages,max_ctas", [(0, 1), (2, 2), (3, 3)])
+def test_s_buffers_handed_round_in_product_order(shape, N, causal, kv_stages, max_ctas):
+    """The tile shapes that leave tensor memory room for more S buffers than Q tiles (d = 64, a single Q tile, 64-row K/V
+    tiles): S of a tile's next step is issued before its present P is waited for, and the buffers go round in the order
+    of the products of both tiles.  Ragged heads make that order irregular: second tiles that lie beyond N for whole
+    items (their MMA lane skips those products and runs ahead), diagonals that end one tile's products a step before the
+    other's, backward scans that start with such a step.  Few CTAs with many items each, shallow K/V rings, static and
+    dynamic schedule, both orders, launches repeated: the result stays the oracle's, and the static one bit for bit."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    d, block_n, q_tiles = shape
+    w = wl.small_workload("s-buffers", 2, 3, N, d, wl.BF16 if d == 128 else wl.F16, causal, 7800 + N)
+    qkv = upload(w)
+    q, k, v = qkv
+    adt = sa.BF16 if d == 128 else sa.F16
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        opts = opts_for(block_n, q_tiles, kv_stages=kv_stages, max_ctas=max_ctas)
+        first = run_cuda(w, qkv, order, opts)
+        assert_parity(w, first)
+        for _ in range(3):
+            assert torch.equal(run_cuda(w, qkv, order, opts).view(torch.int16), first.view(torch.int16))
+        dyn = opts_for(block_n, q_tiles, kv_stages=kv_stages, max_ctas=max_ctas, pairing=1)
+        nb = sa.attn_dynamic_scratch_bytes(max_ctas)
+        scratch = torch.zeros(nb // 4, dtype=torch.int32, device=q.device)
+        for _ in range(2):
+            o = torch.full_like(q, float("nan"))
+            sa.attn_fwd_dynamic(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, int(causal), order,
+                                adt, torch.cuda.current_stream().cuda_stream, dyn, scratch.data_ptr(), nb)
+            sa.attn_device_status()
+            assert_parity(w, o)
+
+
 def test_host_entry_point_from_two_threads():
     """Two host threads, each with its own stream and buffers, call attn_fwd_host at the same time (ctypes drops the
     interpreter lock during the call): the device's one pipeline is handed from call to call under its lock, and both
