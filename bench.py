@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--also c3,c4] [--impl reference]
 
 Prints ONE JSON line.  The workload is c5 (B=2 H=16 N=65536 d=128 bf16 causal), the largest of the five
-configurations; c3, c4, c2 and a d = 64 shape that fills the GPU (d64-n8k) are measured the same way and reported, each
-with its own roofline block, under `also`.
+configurations; c3, c4, c2, a d = 64 shape that fills the GPU (d64-n8k) and the shape of the paper's own sweep (B = 8,
+N = 131072, d = 64, with and without the causal mask) are measured the same way and reported, each with its own roofline
+block, under `also`.
 
 How a workload is timed.  The two scan orders are launched in alternation, cyclic, sawtooth, cyclic, ..., every
 launch between its own pair of CUDA events on the launch stream, after a warm-up of the same alternating launches
@@ -63,6 +64,14 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     ("c5", "sawtooth", "mirrored"): (2469511936, 523371264),
     ("c5", "cyclic", "none"): (5360406272, 533639168),
     ("c5", "sawtooth", "none"): (9153945088, 534020096),
+}
+
+
+# What the paper reports for the two shapes of its sweep that bench.py also times (its Section 4.3, CuTile results, sawtooth
+# order): another machine and another kernel, context for the reader, not a target.
+PAPER_CONTEXT = {
+    "sweep-d64-b8": {"tflops": 69.0, "what": "paper, GB10, CuTile kernel with 64x64 tiles, sawtooth order, B=8 S=131072 D=64 non-causal"},
+    "sweep-d64-b8-causal": {"tflops": 66.0, "what": "paper, GB10, CuTile kernel with 64x64 tiles, sawtooth order, B=8 S=131072 D=64 causal"},
 }
 
 
@@ -449,7 +458,7 @@ def main():
     ap.add_argument("--pairing", default="default", choices=["default", "none", "mirrored", "adjacent"],
                     help="how the static walk groups work items (default: mirrored pairs under the causal mask)")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the persistent grid (the paper's 'active SMs'); 0 = all SMs")
-    ap.add_argument("--also", default="c3,c4,d64-n8k,c2",
+    ap.add_argument("--also", default="c3,c4,d64-n8k,c2,sweep-d64-b8,sweep-d64-b8-causal",
                     help="further workloads measured the same way (single GPU only; '' for none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (default: min(steps, 5))")
@@ -522,6 +531,8 @@ def main():
             if only is None:
                 blk["dynamic_schedule"] = bench.dynamic_leg(wk, dv, ln, headline, 5)
             blk["steps"] = n_steps
+            if name in PAPER_CONTEXT:
+                blk["paper_context"] = dict(PAPER_CONTEXT[name], ratio=blk["tflops"] / PAPER_CONTEXT[name]["tflops"])
             also[name] = blk
             del dv, ln
             torch.cuda.empty_cache()

@@ -81,6 +81,8 @@ STUDY_CASES = {
 for _b in (1, 2, 4, 8):
     STUDY_CASES[f"sweep-d64-b{_b}"] = Workload(f"sweep-d64-b{_b}", _b, 1, 131072, 64, F16, False, 2100 + _b)
     STUDY_CASES[f"sweep-d128-b{_b}"] = Workload(f"sweep-d128-b{_b}", _b, 1, 131072, 128, BF16, False, 2200 + _b)
+# The same shape under the causal mask (the paper's second CuTile result).
+STUDY_CASES["sweep-d64-b8-causal"] = Workload("sweep-d64-b8-causal", 8, 1, 131072, 64, F16, True, 2300)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
