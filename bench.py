@@ -54,16 +54,16 @@ WARMUP_LOAD_SECONDS = 0.25
 # kernel on the full-size workload with the default launch plan (three metrics, one pass).
 # Keyed by (workload, scan order, pairing in force); anything else reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "cyclic", "none"): (403255040, 116423936),
-    ("c3", "sawtooth", "none"): (404629248, 115891712),
-    ("c4", "cyclic", "mirrored"): (980670976, 252060416),
-    ("c4", "sawtooth", "mirrored"): (947037184, 250663424),
-    ("c4", "cyclic", "none"): (1358940928, 260275968),
-    ("c4", "sawtooth", "none"): (1982593280, 259297792),
-    ("c5", "cyclic", "mirrored"): (2706657792, 523120384),
-    ("c5", "sawtooth", "mirrored"): (2469511936, 523371264),
-    ("c5", "cyclic", "none"): (5360406272, 533639168),
-    ("c5", "sawtooth", "none"): (9153945088, 534020096),
+    ("c3", "cyclic", "none"): (404312832, 113961984),
+    ("c3", "sawtooth", "none"): (406504192, 114424576),
+    ("c4", "cyclic", "mirrored"): (968785152, 250669568),
+    ("c4", "sawtooth", "mirrored"): (974485504, 251215616),
+    ("c4", "cyclic", "none"): (1200302336, 258832896),
+    ("c4", "sawtooth", "none"): (1640605184, 259677952),
+    ("c5", "cyclic", "mirrored"): (2634280960, 521590528),
+    ("c5", "sawtooth", "mirrored"): (2511834112, 526502400),
+    ("c5", "cyclic", "none"): (5354950144, 535655936),
+    ("c5", "sawtooth", "none"): (7901230592, 532906240),
 }
 
 
