@@ -164,3 +164,19 @@ def test_host_groups():
         sa.attn_host_groups(0, mib)
     with pytest.raises(sa.AttnError):
         sa.attn_host_groups(4, mib, 33)
+
+
+def test_measuring_aids_compile():
+    """The two stand-alone measuring aids at the repository root compile for sm_100a against the in-tree headers and
+    library (they are run on a GPU by hand or by bench.py, never here)."""
+    import subprocess
+    import tempfile
+    from conftest import nvcc_available
+    if not nvcc_available():
+        pytest.skip("nvcc not found")
+    from paper_2601_16032_b200 import build as lib_build
+    assert os.path.exists(lib_build.build_host_call_probe())
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with tempfile.TemporaryDirectory() as tmp:
+        subprocess.run([os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc"), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a",
+                        "-o", os.path.join(tmp, "profile_mma_rate"), os.path.join(root, "profile_mma_rate.cu")], check=True, cwd=root)
