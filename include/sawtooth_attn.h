@@ -142,8 +142,10 @@ int attn_fwd_ex(const void* q, const void* k, const void* v, void* o,
  * persistent loop hands CTA c the items c, c+G, ...; under the causal mask those differ in length by up to the whole
  * sequence, and CTAs that drew short ones idle at the end).  Here every persistent CTA claims its next work item from
  * a counter in `scratch`, in index order, which under the causal mask runs from the longest Q block of a head to the
- * shortest.  Algorithm 4's alternation still follows the CTA's own count of items, so which items a CTA scans
- * backward depends on the race for the counter: results are reproducible bit for bit in the cyclic order only.
+ * shortest.  Algorithm 4's alternation follows the round of a claim (claim index / grid size): that is the CTA's own
+ * count of items as long as the CTAs stay in step, and it does not depend on which CTA won the claim, so for fixed
+ * arguments the result is reproducible bit for bit in both scan orders although the assignment of items to CTAs is not
+ * (without the causal mask it is the static, unpaired schedule's result).
  *
  * scratch: DEVICE memory owned by the caller, 4-byte aligned, at least attn_dynamic_scratch_bytes(plan.grid) bytes
  * (plan from attn_query_plan with opts->pairing = ATTN_PAIR_NONE, since single items are claimed here;

@@ -232,7 +232,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // units blockIdx.x, += gridDim.x; `slot` counts the positions of that walk (a unit holds one or two items).
     // Dynamic schedule: the producer warp claims the next unclaimed item from a global counter and passes it to the
     // other roles through a two-slot mailbox in shared memory, so a CTA that drew short items simply draws more of
-    // them.  Algorithm 4's parity is the CTA's own count `it` either way.
+    // them.  Algorithm 4's parity is the CTA's own count `it` on the static walk and the claim's round on the dynamic one.
     const bool dynamic = p.work_counter != nullptr;
     auto static_next = [&](int& slot, int it, WorkItem& w) -> bool {
         for (;;) {
@@ -242,8 +242,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     };
     auto claimed_item = [&](long long claim, int it) -> WorkItem {
+        // The scan direction of a claimed item follows the round of its claim (claim index / grid size): the CTA's own
+        // count while the CTAs stay in step, and independent of which CTA won the claim, so results are reproducible.
+        (void)it;
         const Slot sl = claimed_slot(p.sched, claim);
-        return make_item(p.sched, sl.bh, sl.q_item, it);
+        return make_item(p.sched, sl.bh, sl.q_item, (int)(claim / (long long)gridDim.x));
     };
     auto claim_work = [&](int it, bool& ok) -> long long {  // producer warp, all lanes (dynamic schedule)
         const int slot = it & 1;

@@ -1,6 +1,7 @@
 """GPU tests of attn_fwd_dynamic: the persistent CTAs claim their work items from a counter in caller-provided
 scratch memory instead of walking Algorithm 2's fixed grid-stride sequence.  The result must be the oracle's, every
-item must be handled exactly once, and in the cyclic order the output must equal the static schedule's bit for bit."""
+item must be handled exactly once, the output must be the same launch after launch, and in the cyclic order it must
+equal the static schedule's bit for bit."""
 import numpy as np
 import pytest
 
@@ -68,6 +69,33 @@ def test_dynamic_cyclic_equals_static_bitwise():
                 torch.cuda.current_stream().cuda_stream)
     sa.attn_device_status()
     assert torch.equal(o_dyn.view(torch.int16), o_sta.view(torch.int16))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_dynamic_sawtooth_is_reproducible(causal):
+    """Which CTA wins a claim is a race, but an item's scan direction follows the round of its claim, not the winner's own
+    count: launch after launch gives the same bits, with few CTAs (many claims each) and with one per item's worth of SMs;
+    without the causal mask they are the bits of the static, unpaired schedule."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    w = wl.small_workload("dyn-repro", 2, 3, 1700, 128, wl.BF16, causal, 7550)
+    q, k, v = qkv = upload(w)
+    for max_ctas in (3, 0):
+        opts = sa.Opts()
+        opts.max_ctas = max_ctas
+        first, _, _ = run_dynamic(w, qkv, sa.SAWTOOTH, opts)
+        assert_parity(w, first)
+        for _ in range(5):
+            again, _, _ = run_dynamic(w, qkv, sa.SAWTOOTH, opts)
+            assert torch.equal(again.view(torch.int16), first.view(torch.int16))
+        if not causal:
+            sta = sa.Opts()
+            sta.max_ctas, sta.pairing = max_ctas, sa.PAIR_NONE
+            o_sta = torch.empty_like(q)
+            sa.attn_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o_sta.data_ptr(), w.B, w.H, w.N, w.d, w.scale, 0, sa.SAWTOOTH, sa.BF16,
+                           torch.cuda.current_stream().cuda_stream, sta)
+            sa.attn_device_status()
+            assert torch.equal(first.view(torch.int16), o_sta.view(torch.int16))
 
 
 def test_dynamic_rejects_bad_scratch_and_launch_mode():
