@@ -230,6 +230,16 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
                         attn_trace_entry* buf, size_t cap, size_t* n);
 
 /*
+ * Host-only replay of the dynamic schedule (attn_fwd_dynamic): the work items in the order in which they are claimed,
+ * each with the scan direction that the round of its claim gives it.  Which CTA takes a claim is not determined:
+ * entries carry cta = -1, iteration = the round (claim index / grid size), k = the claim index, member = 0.
+ * Arguments as for attn_schedule_trace; opts->pairing is ignored.
+ */
+int attn_dynamic_claim_trace(int B, int H, int N, int d, int causal, int scan_order, int dtype,
+                             const attn_fwd_opts* opts, int sm_count,
+                             attn_trace_entry* buf, size_t cap, size_t* n);
+
+/*
  * Waits for the current device and reads, then clears, its kernel status word: 0, or a code naming
  * the wait that ran out in a kernel launched since the last call.  Returns ATTN_OK when the word
  * was 0, ATTN_ERR_DEVICE_TIMEOUT otherwise (code in *code if code != NULL).

@@ -22,6 +22,12 @@ scans about t+1 tiles' worth of K/V, so the two members of a mirrored pair scan 
 whatever p is, and all units take the same time.  An odd middle tile forms a unit of its own.
 i_local still counts Q tiles, so in the sawtooth order the first member of a pair is scanned
 forward and the second backward.
+
+Dynamic claims (a variant of Algorithm 2 in which a CTA takes the next unclaimed index from a shared
+counter instead of adding G to its own): claim c = 0, 1, 2, ... names the Q tile that linear index c
+names, except that under the causal mask the tiles of a head are handed out from the last (longest
+scan) to the first.  Which CTA gets a claim is not determined; the scan direction is, by the round
+of the claim, c // G: the value i_local would have if the CTAs took their claims in turn.
 """
 from __future__ import annotations
 
@@ -118,3 +124,19 @@ def full_schedule(n_sm: int, B: int, H: int, N: int, W: int, B_c: int, causal: b
     n_units = B * H * units_per_head(ceil_div(N, W), pairing)
     G = grid_size(n_units, n_sm if max_ctas <= 0 else min(n_sm, max_ctas))
     return [list(cta_sequence(c, G, B, H, N, W, B_c, causal, scan_order, digit_order, pairing)) for c in range(G)]
+
+
+def dynamic_claims(n_sm: int, B: int, H: int, N: int, W: int, B_c: int, causal: bool, scan_order: int,
+                   digit_order: str = "tile_fastest", max_ctas: int = 0) -> list[WorkItem]:
+    """The Q tiles in the order in which the dynamic schedule hands them out (cta = -1: not determined)."""
+    n_q = ceil_div(N, W)
+    n_work = B * H * n_q
+    G = grid_size(n_work, n_sm if max_ctas <= 0 else min(n_sm, max_ctas))
+    out = []
+    for c in range(n_work):
+        b, h, pos = decode(c, B, H, n_q, digit_order)
+        t = n_q - 1 - pos if causal else pos
+        rnd = c // G
+        backward = scan_order == SAWTOOTH and rnd % 2 == 1
+        out.append(WorkItem(-1, rnd, c, b, h, t, backward, kv_tiles_needed(t, N, W, B_c, causal)))
+    return out

@@ -7,7 +7,7 @@ is no CPU fallback: without the built library, or without a B200, the calls rais
 from .binding import (  # noqa: F401
     CYCLIC, SAWTOOTH, F16, BF16, TILE_FASTEST, HEAD_FASTEST, PAIR_DEFAULT, PAIR_NONE, PAIR_MIRRORED, PAIR_ADJACENT, LAYOUT_BHND, LAYOUT_BNHD,
     AttnError, Opts, Plan, TraceEntry,
-    attn_fwd, attn_fwd_ex, attn_fwd_dynamic, attn_fwd_dynamic_noalloc, attn_dynamic_scratch_bytes, attn_fwd_host, attn_host_groups, attn_query_plan, attn_schedule_trace,
+    attn_fwd, attn_fwd_ex, attn_fwd_dynamic, attn_fwd_dynamic_noalloc, attn_dynamic_scratch_bytes, attn_fwd_host, attn_host_groups, attn_query_plan, attn_schedule_trace, attn_dynamic_claim_trace,
     attn_device_status, attn_last_kernel_cycles, attn_status_string, attn_last_error, library_path, load_library,
     forward,
 )

@@ -78,6 +78,8 @@ def load_library():
                                                 ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     lib.attn_host_groups.argtypes = [ctypes.c_longlong, ctypes.c_size_t, ci, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ci)]
     lib.attn_host_groups.restype = ci
+    lib.attn_dynamic_claim_trace.argtypes = lib.attn_schedule_trace.argtypes
+    lib.attn_dynamic_claim_trace.restype = ci
     lib.attn_device_status.argtypes = [ctypes.POINTER(ci)]
     lib.attn_last_kernel_cycles.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
     lib.attn_last_kernel_cycles.restype = ci
@@ -161,6 +163,16 @@ def attn_schedule_trace(B: int, H: int, N: int, d: int, causal: int, scan_order:
     _check(lib.attn_schedule_trace(B, H, N, d, int(causal), scan_order, dtype, _opts_ptr(opts), sm_count, None, 0, ctypes.byref(n)))
     buf = (TraceEntry * n.value)()
     _check(lib.attn_schedule_trace(B, H, N, d, int(causal), scan_order, dtype, _opts_ptr(opts), sm_count, buf, n.value, ctypes.byref(n)))
+    return list(buf)
+
+
+def attn_dynamic_claim_trace(B: int, H: int, N: int, d: int, causal: int, scan_order: int, dtype: int,
+                             opts: Optional[Opts] = None, sm_count: int = 0) -> list:
+    lib = load_library()
+    n = ctypes.c_size_t(0)
+    _check(lib.attn_dynamic_claim_trace(B, H, N, d, int(causal), scan_order, dtype, _opts_ptr(opts), sm_count, None, 0, ctypes.byref(n)))
+    buf = (TraceEntry * n.value)()
+    _check(lib.attn_dynamic_claim_trace(B, H, N, d, int(causal), scan_order, dtype, _opts_ptr(opts), sm_count, buf, n.value, ctypes.byref(n)))
     return list(buf)
 
 

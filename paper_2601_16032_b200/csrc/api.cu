@@ -374,6 +374,47 @@ int attn_schedule_trace(int B, int H, int N, int d, int causal, int scan_order, 
     return ATTN_OK;
 }
 
+int attn_dynamic_claim_trace(int B, int H, int N, int d, int causal, int scan_order, int dtype, const attn_fwd_opts* opts,
+                             int sm_count, attn_trace_entry* buf, size_t cap, size_t* n) {
+    if (!n) return fail(ATTN_ERR_INVALID_ARG, "n is null");
+    if (cap > 0 && !buf) return fail(ATTN_ERR_INVALID_ARG, "buf is null");
+    if (scan_order != ATTN_SCAN_CYCLIC && scan_order != ATTN_SCAN_SAWTOOTH)
+        return fail(ATTN_ERR_INVALID_ARG, "unknown scan_order %d", scan_order);
+    attn_fwd_opts single;
+    memset(&single, 0, sizeof(single));
+    if (opts) single = *opts;
+    single.pairing = ATTN_PAIR_NONE;   // single items are claimed
+    attn_plan plan;
+    int rc = attn_query_plan(B, H, N, d, causal, dtype, &single, sm_count, &plan);
+    if (rc) return rc;
+    const SchedParams sp = make_sched(B, H, N, plan.q_tiles, plan.block_n, causal, scan_order == ATTN_SCAN_SAWTOOTH,
+                                      single.digit_order == ATTN_HEAD_FASTEST, causal ? 1 : 0, kPairNone);
+    size_t count = 0;
+    for (long long claim = 0;; ++claim) {
+        const Slot sl = claimed_slot(sp, claim);
+        if (sl.kind == kSlotEnd) break;
+        if (count < cap) {
+            const int round = (int)(claim / plan.grid);
+            const WorkItem w = make_item(sp, sl.bh, sl.q_item, round);
+            attn_trace_entry* e = &buf[count];
+            e->cta = -1;
+            e->iteration = round;
+            e->k = claim;
+            e->batch = w.bh / H;
+            e->head = w.bh % H;
+            e->q_item = w.q_item;
+            e->backward = w.backward;
+            e->n_kv = w.hi;
+            e->n_kv_q0 = w.hi_q[0];
+            e->n_kv_q1 = w.hi_q[1];
+            e->member = 0;
+        }
+        ++count;
+    }
+    *n = count;
+    return ATTN_OK;
+}
+
 static int fwd_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, float scale, int causal,
                       int scan_order, int dtype, void* stream, const attn_fwd_opts* opts, int* work_counter, size_t counter_bytes,
                       int counter_ctas_max);

@@ -142,6 +142,34 @@ def check_replay(n_sm, B, H, N, d, q_tiles, block_n, causal, order, digits, pair
         assert max(g.n_kv_q0, g.n_kv_q1) == g.n_kv
 
 
+@pytest.mark.parametrize("n_sm,max_ctas", [(148, 0), (148, 3), (5, 0)])
+@pytest.mark.parametrize("B,H,N,q_tiles,block_n", [(2, 3, 1330, 2, 128), (1, 5, 700, 1, 64), (3, 1, 256, 2, 128), (1, 2, 4096, 2, 128)])
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("order", [0, 1])
+@pytest.mark.parametrize("digits", [0, 1])
+def test_dynamic_claim_replay_equals_the_schedule_oracle(n_sm, max_ctas, B, H, N, q_tiles, block_n, causal, order, digits):
+    """The dynamic schedule's order of claims: the linear order of Algorithm 2, the Q blocks of a head from the longest
+    scan to the shortest under the causal mask, the direction of a block from the round of its claim."""
+    o = sa.Opts()
+    o.q_tiles, o.block_n, o.digit_order, o.max_ctas = q_tiles, block_n, digits, max_ctas
+    got = sa.attn_dynamic_claim_trace(B, H, N, 128, causal, order, sa.BF16, o, sm_count=n_sm)
+    W = 128 * q_tiles
+    want = sch.dynamic_claims(n_sm, B, H, N, W, block_n, bool(causal), order, "head_fastest" if digits else "tile_fastest", max_ctas)
+    assert len(got) == len(want) == B * H * -(-N // W)
+    for g, w in zip(got, want):
+        assert (g.cta, g.iteration, g.k, g.batch, g.head, g.q_item, bool(g.backward), g.n_kv, g.member) == \
+            (-1, w.i_local, w.k, w.batch, w.head, w.q_tile, w.backward, w.n_kv, 0)
+    assert sorted((g.batch, g.head, g.q_item) for g in got) == sorted((b, h, t) for b in range(B) for h in range(H) for t in range(-(-N // W)))
+    if causal and not digits:   # within a head the scans never get longer
+        for a, b in zip(got, got[1:]):
+            if (a.batch, a.head) == (b.batch, b.head):
+                assert a.n_kv >= b.n_kv
+    if not causal and max_ctas == 0:   # the static, unpaired walk hands out the same blocks with the same directions
+        o.pairing = sa.PAIR_NONE
+        static = {(e.batch, e.head, e.q_item): bool(e.backward) for e in sa.attn_schedule_trace(B, H, N, 128, 0, order, sa.BF16, o, sm_count=n_sm)}
+        assert static == {(g.batch, g.head, g.q_item): bool(g.backward) for g in got}
+
+
 def test_host_groups():
     """attn_fwd_host's groups of heads: equal ones on request; left to the library, one group for small tensors and
     otherwise one per 16 MiB of a tensor, 32 at most, a head at least."""
