@@ -1,5 +1,6 @@
 """GPU parity on the five benchmark configurations at full size, through the C ABI, in the launch
-configuration the benchmark times (library defaults), both scan orders.
+configuration the benchmark times (library defaults), both scan orders; for c3, c4 and c5 also on the dynamic schedule
+of the benchmark's second leg, for c5 also through attn_fwd_host, its end-to-end leg.
 
 The oracle result of the checked rows is computed once per configuration and both orders are
 compared with it: every row of every head for c1 and c2, every row of two heads plus seeded rows
@@ -13,7 +14,7 @@ from parity_util import MAX_ABS_TOL, MEAN_ABS_TOL, oracle_rows, compare_rows, ru
 pytestmark = pytest.mark.gpu
 
 
-def check_config(name, opts_list):
+def check_config(name, opts_list, also_dynamic=False, also_host=False):
     import torch
     import paper_2601_16032_b200 as sa
     w = wl.CONFIGS[name]
@@ -29,6 +30,37 @@ def check_config(name, opts_list):
                 f"{name} {label} order {order}: max_abs {max_abs:.3e} mean_abs {mean_abs:.3e} over {n_rows} rows"
             outs[(label, order)] = o if w.compulsory_bytes <= (64 << 20) else None
             del o
+    if also_dynamic or also_host:
+        q, k, v = qkv
+        adt = sa.BF16 if w.dtype == wl.BF16 else sa.F16
+        stream = torch.cuda.current_stream().cuda_stream
+        o = torch.empty_like(q)
+    if also_dynamic:   # the schedule of the benchmark's second leg
+        single = sa.Opts()
+        single.pairing = sa.PAIR_NONE
+        n_bytes = sa.attn_dynamic_scratch_bytes(sa.attn_query_plan(w.B, w.H, w.N, w.d, int(w.causal), adt, single).grid)
+        scratch = torch.zeros(n_bytes // 4, dtype=torch.int32, device=q.device)
+        for order in (sa.CYCLIC, sa.SAWTOOTH):
+            o.fill_(float("nan"))
+            sa.attn_fwd_dynamic(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, int(w.causal), order, adt,
+                                stream, None, scratch.data_ptr(), n_bytes)
+            sa.attn_device_status()
+            max_abs, mean_abs, n_rows = compare_rows(w, o, plan, want)
+            assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, f"{name} dynamic order {order}: max_abs {max_abs:.3e} mean_abs {mean_abs:.3e}"
+    if also_host:      # the benchmark's end-to-end leg: host buffers in and out, the library's own groups of heads
+        host = [t.view(torch.int16).cpu().pin_memory() for t in (q, k, v)]
+        o_host = torch.full(q.shape, -1, dtype=torch.int16).pin_memory()
+        staging = [torch.empty_like(q) for _ in range(3)]
+        o.fill_(float("nan"))
+        sa.attn_fwd_host(host[0].data_ptr(), host[1].data_ptr(), host[2].data_ptr(), o_host.data_ptr(), staging[0].data_ptr(),
+                         staging[1].data_ptr(), staging[2].data_ptr(), o.data_ptr(), w.B, w.H, w.N, w.d, w.scale, int(w.causal), sa.SAWTOOTH,
+                         adt, stream, None)
+        torch.cuda.synchronize()
+        sa.attn_device_status()
+        got = o_host.view(q.dtype).cuda()
+        max_abs, mean_abs, n_rows = compare_rows(w, got, plan, want)
+        assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, f"{name} host entry point: max_abs {max_abs:.3e} mean_abs {mean_abs:.3e}"
+        del host, o_host, staging, got
     torch.cuda.empty_cache()
     return w, outs
 
@@ -51,15 +83,15 @@ def test_c2_all_rows_128x64_tiles_and_default():
 
 
 def test_c3_two_heads_plus_sampled_rows():
-    check_config("c3", [("default", None)])
+    check_config("c3", [("default", None)], also_dynamic=True)
 
 
 def test_c4_causal_two_heads_plus_sampled_rows():
-    check_config("c4", [("default", None)])
+    check_config("c4", [("default", None)], also_dynamic=True)
 
 
 def test_c5_causal_sampled_rows_every_head():
-    check_config("c5", [("default", None)])
+    check_config("c5", [("default", None)], also_dynamic=True, also_host=True)
 
 
 def test_long_single_head_beyond_l2_sampled_rows():
