@@ -118,6 +118,21 @@ def test_long_single_head_beyond_l2_sampled_rows():
     assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, ("dynamic", max_abs, mean_abs, n_rows)
 
 
+@pytest.mark.parametrize("name", ["d64-n8k", "sweep-d64-b8", "sweep-d64-b8-causal"])
+def test_d64_benchmark_shapes_sampled_rows(name):
+    """The d = 64 shapes the benchmark also times (a shape that fills the GPU, and the paper's own sweep shape with and
+    without the causal mask: 512 K/V steps per work item through three S buffers): seeded rows of every head, both orders."""
+    import paper_2601_16032_b200 as sa
+    w = wl.STUDY_CASES[name]
+    plan = {bh: wl.sampled_rows(w, bh[0], bh[1], 96 if w.N > 10000 else 24) for bh in wl.all_heads(w)}
+    want = oracle_rows(w, plan)
+    qkv = upload(w)
+    for order in (sa.CYCLIC, sa.SAWTOOTH):
+        o = run_cuda(w, qkv, order)
+        max_abs, mean_abs, n_rows = compare_rows(w, o, plan, want)
+        assert max_abs <= MAX_ABS_TOL and mean_abs <= MEAN_ABS_TOL, (name, order, max_abs, mean_abs, n_rows)
+
+
 def test_many_small_heads():
     """1,500 heads of 300 keys: many more (batch, head) pairs than SMs, ragged length, both tile shapes."""
     import paper_2601_16032_b200 as sa
