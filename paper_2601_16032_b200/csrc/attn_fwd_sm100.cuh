@@ -560,7 +560,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // ------------------------------------------------------------------ softmax / correction / epilogue
         if (G::kRebalance) ptx::reg_alloc<G::kRegsSoftmax>();
         constexpr int kColsS = G::kColsS, kColsO = G::kColsO;
-        constexpr int kExpPolyMask = kD == 64 ? SAW_EXP_POLY_MASK_D64 : SAW_EXP_POLY_MASK_D128;
+        // (Measured per tile shape: with 64-row K/V tiles at d = 64 three pairs in eight, with a single Q tile at d = 128,
+        // where the softmax sets the step as well, one in eight.)
+        constexpr int kExpPolyMask = kD == 64 ? (kBlockN == 64 ? 0x49 : SAW_EXP_POLY_MASK_D64)
+                                              : (kQTiles == 1 ? 0x01 : SAW_EXP_POLY_MASK_D128);
         const int q = warp >> 2;                       // which Q tile this thread works on
         const int r_in_tile = (warp & 3) * 32 + lane;  // row inside the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
