@@ -127,6 +127,9 @@ typedef struct {
  * The forward pass (Eq. 1 via Algorithms 1, 2, 4).  q, k, v, o: DEVICE pointers, layout as above.
  * causal: 0 or 1.  scan_order: attn_scan_order.  dtype: attn_dtype.  stream: a cudaStream_t (NULL =
  * the default stream).  Asynchronous.  `o` is fully overwritten.
+ * A device's first call also looks up the library's device symbols and raises the kernel's shared-memory limit; every
+ * later call (attn_fwd_ex without check_mode and attn_fwd_dynamic likewise) only enqueues work on `stream`, so it may be
+ * captured into a CUDA graph and replayed.
  */
 int attn_fwd(const void* q, const void* k, const void* v, void* o,
              int B, int H, int N, int d, float scale, int causal, int scan_order,

@@ -387,6 +387,64 @@ def test_s_buffers_handed_round_in_product_order(shape, N, causal, kv_stages, ma
             assert_parity(w, o)
 
 
+def test_calls_captured_in_a_cuda_graph_replay_bit_for_bit():
+    """After one call outside any capture (the library looks its device symbols up and raises the kernel's shared-memory
+    limit on a device's first call), attn_fwd, attn_fwd_ex with a log-sum-exp output and attn_fwd_dynamic only enqueue
+    work on the stream they are given: captured into a CUDA graph and replayed on new inputs in the same buffers, they
+    give what the direct calls give."""
+    import torch
+    import paper_2601_16032_b200 as sa
+    wa = wl.small_workload("graph-a", 1, 3, 1100, 128, wl.BF16, True, 7950)
+    wb = wl.small_workload("graph-b", 1, 3, 1100, 128, wl.BF16, True, 7951)
+    a, b = upload(wa), upload(wb)
+    q, k, v = (torch.empty_like(t) for t in a)
+    o1, o2, o3 = (torch.empty_like(q) for _ in range(3))
+    lse = torch.empty((wa.B, wa.H, wa.N), dtype=torch.float32, device=q.device)
+    opts = sa.Opts()
+    opts.lse = lse.data_ptr()
+    single = sa.Opts()
+    single.pairing = sa.PAIR_NONE
+    nb = sa.attn_dynamic_scratch_bytes(sa.attn_query_plan(wa.B, wa.H, wa.N, wa.d, 1, sa.BF16, single).grid)
+    scratch = torch.zeros(nb // 4, dtype=torch.int32, device=q.device)
+
+    def calls(stream):
+        args = (q.data_ptr(), k.data_ptr(), v.data_ptr())
+        shape = (wa.B, wa.H, wa.N, wa.d, wa.scale, 1, sa.SAWTOOTH, sa.BF16, stream)
+        sa.attn_fwd(*args, o1.data_ptr(), *shape)
+        sa.attn_fwd_ex(*args, o2.data_ptr(), *shape, opts)
+        sa.attn_fwd_dynamic(*args, o3.data_ptr(), *shape, None, scratch.data_ptr(), nb)
+
+    for dst, src in zip((q, k, v), a):
+        dst.copy_(src)
+    calls(torch.cuda.current_stream().cuda_stream)     # the first calls on the device, outside the capture
+    torch.cuda.synchronize()
+    sa.attn_device_status()
+    want_a = [t.clone() for t in (o1, o2, o3, lse)]
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            calls(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.current_stream().wait_stream(side)
+    for inputs, want in ((b, None), (a, want_a)):
+        for dst, src in zip((q, k, v), inputs):
+            dst.copy_(src)
+        for t in (o1, o2, o3):
+            t.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        sa.attn_device_status()
+        if want is None:
+            assert_parity(wb, o1)
+            assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+            assert_parity(wb, o3)
+        else:
+            for got, w_ in zip((o1, o2, o3), want[:3]):
+                assert torch.equal(got.view(torch.int16), w_.view(torch.int16))
+            assert torch.equal(lse, want[3])
+
+
 def test_host_entry_point_from_two_threads():
     """Two host threads, each with its own stream and buffers, call attn_fwd_host at the same time (ctypes drops the
     interpreter lock during the call): the device's one pipeline is handed from call to call under its lock, and both
